@@ -1,0 +1,254 @@
+"""fp64 CPU oracle of the AdaPM optimizer step.  TEST INFRASTRUCTURE ONLY.
+
+This file is the slow, plain definition the CUDA library is checked against.
+It is written from the paper's Algorithm 1 (low-rank update with correction),
+Algorithm 2 (gradient-descent refit of the factors), Eq. 4 (full momentum) and
+the Adam-mini combination of Section 5.1.3 / Related Work (one second-moment
+scalar per parameter group = the group average of Adam's statistic).  It shares
+no code with the CUDA path, imports nothing from it, and only the tests, the
+smoke check and the benchmark's CPU-baseline leg may call it.
+
+Everything is float64.  Inputs are the exact values the device receives
+(fp32 parameters, fp32 or bf16-rounded gradients) widened to float64.
+
+Readings of the paper taken here (each is a choice; the paper does not settle it):
+  * Algorithm 1's last line prints "lambda x_t"; x_t is read as W_t
+    (decoupled weight decay).
+  * clip(., 1) is the elementwise clamp of the ratio to [-1, 1].
+  * No 1/(1-beta^t) debiasing appears in Algorithm 1, so none is applied
+    unless `adam_debias` is set (used only to compare with textbook AdamW).
+  * Algorithm 2 evaluates both partial derivatives at the same (L, R) and
+    then updates both factors (simultaneous, not alternating).
+  * The step sizes eta_k = 0.5 (1 + cos(pi k / K)), k = 1..K, are absolute;
+    eta_K = 0, so the K-th pass changes nothing.
+  * L_0 = R_0 = 0 is a stationary point of Algorithm 2 (both derivatives are
+    zero there), so the factors would never move.  R_0 = 0 is kept (L_0 R_0 = 0,
+    hence m_1 is unchanged) and L_0 is given orthonormal columns: Gaussian draws
+    orthonormalised by modified Gram-Schmidt, rounded to fp32 (`init_L0`).
+  * "No momentum" blocks use m^c_t = g_t.
+Parity with the authors' unreleased code on these readings is unpinned; what is
+pinned (tests/test_oracle_pins.py) is this oracle against closed forms, special
+cases, a library optimizer, the proof identity of Theorem 2 and brute force.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional
+
+import numpy as np
+
+MOM_NONE = 0
+MOM_FULL = 1
+MOM_LOWRANK = 2
+V_ELEMENT = 0
+V_BLOCKMEAN = 1
+
+
+@dataclass
+class Block:
+    """One parameter block W in R^{rows x cols} and how it is treated."""
+    rows: int
+    cols: int
+    mom_mode: int = MOM_FULL
+    rank: int = 0
+    v_mode: int = V_ELEMENT
+    v_group_rows: int = 0        # BLOCKMEAN: consecutive rows per group; 0 = the whole block
+    lr_scale: float = 1.0
+    weight_decay: float = 0.0
+    offset: int = 0              # element offset in a flat buffer (bookkeeping only)
+
+    def n_groups(self) -> int:
+        if self.v_mode == V_ELEMENT:
+            return self.rows * self.cols
+        return 1 if self.v_group_rows == 0 else self.rows // self.v_group_rows
+
+
+@dataclass
+class HParams:
+    lr: float = 1e-3
+    beta1: float = 0.9
+    beta2: float = 0.95
+    eps: float = 1e-8
+    clip: float = 1.0            # math.inf disables the clamp
+    inner_iters: int = 5         # K of Algorithm 2
+    inner_lr_scale: float = 1.0  # multiplies every eta_k; 1 = as printed
+    adam_debias: bool = False
+    correction: bool = True      # Eq. 3 on; off: m^c := m_t
+
+
+@dataclass
+class BlockState:
+    m: Optional[np.ndarray] = None   # full momentum m^f (FULL blocks)
+    L: Optional[np.ndarray] = None   # rows x rank
+    R: Optional[np.ndarray] = None   # rank x cols
+    v: Optional[np.ndarray] = None   # rows x cols, or one value per group
+    last: Dict[str, np.ndarray] = field(default_factory=dict)   # transients of the last step
+
+
+# ----------------------------------------------------------------------------------------------
+# Algorithm 2 (Appendix B): K gradient-descent passes on || L R - m_t ||_F^2
+# ----------------------------------------------------------------------------------------------
+
+def inner_schedule(K: int) -> List[float]:
+    """eta_k = 0.5 (1 + cos(pi k / K)) for k = 1..K (Appendix B, text below Algorithm 2)."""
+    return [0.5 * (1.0 + math.cos(math.pi * k / K)) for k in range(1, K + 1)]
+
+
+def lowrank_refit_gd(m_t: np.ndarray, L_prev: np.ndarray, R_prev: np.ndarray, K: int,
+                     scale: float = 1.0):
+    """Algorithm 2: warm start at (L_{t-1}, R_{t-1}); both derivatives from the same point."""
+    L = np.array(L_prev, dtype=np.float64, copy=True)
+    R = np.array(R_prev, dtype=np.float64, copy=True)
+    if K <= 0:
+        return L, R
+    for eta in inner_schedule(K):
+        E = L @ R - m_t                  # L R - m_t
+        dL = E @ R.T                     # dl/dL = (L R - m_t) R^T
+        dR = L.T @ E                     # dl/dR = L^T (L R - m_t)
+        L = L - (scale * eta) * dL
+        R = R - (scale * eta) * dR
+    return L, R
+
+
+def lowrank_refit_exact(m_t: np.ndarray, r: int):
+    """A true minimiser of Eq. 1: the rank-r truncated SVD (Eckart-Young).  Used only by pins."""
+    U, S, Vt = np.linalg.svd(m_t, full_matrices=False)
+    return U[:, :r] * S[:r], Vt[:r, :]
+
+
+def init_L0(rows: int, rank: int, seed: int, block_index: int) -> np.ndarray:
+    """Orthonormal-column L_0: Gaussian draws, modified Gram-Schmidt in fp64, rounded to fp32."""
+    key = np.array([(0xAD0A << 32) | (seed & 0xFFFFFFFF), block_index & 0xFFFFFFFFFFFFFFFF], dtype=np.uint64)
+    G = np.random.Generator(np.random.Philox(key=key)).standard_normal((rows, rank))
+    Q = np.zeros_like(G)
+    for j in range(rank):
+        q = G[:, j].copy()
+        for i in range(j):
+            q -= (Q[:, i] @ q) * Q[:, i]
+        Q[:, j] = q / math.sqrt(q @ q)
+    return Q.astype(np.float32).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------------------------
+# Second-order statistic: Algorithm 1 line 7, or its group average (Adam-mini combination)
+# ----------------------------------------------------------------------------------------------
+
+def second_moment(v_prev: np.ndarray, g: np.ndarray, blk: Block, beta2: float) -> np.ndarray:
+    if blk.v_mode == V_ELEMENT:
+        return beta2 * v_prev + (1.0 - beta2) * (g * g)
+    gr = blk.rows if blk.v_group_rows == 0 else blk.v_group_rows
+    assert blk.rows % gr == 0, "v_group_rows must divide rows"
+    mean_sq = (g * g).reshape(blk.rows // gr, gr * blk.cols).mean(axis=1)
+    return beta2 * v_prev + (1.0 - beta2) * mean_sq
+
+
+def _v_per_element(v: np.ndarray, blk: Block) -> np.ndarray:
+    if blk.v_mode == V_ELEMENT:
+        return v
+    gr = blk.rows if blk.v_group_rows == 0 else blk.v_group_rows
+    return np.repeat(v, gr)[:, None] * np.ones((1, blk.cols))
+
+
+# ----------------------------------------------------------------------------------------------
+# One step of one block
+# ----------------------------------------------------------------------------------------------
+
+def new_state(blk: Block, L0: Optional[np.ndarray] = None) -> BlockState:
+    st = BlockState()
+    if blk.v_mode == V_ELEMENT:
+        st.v = np.zeros((blk.rows, blk.cols))
+    else:
+        st.v = np.zeros(blk.n_groups())
+    if blk.mom_mode == MOM_FULL:
+        st.m = np.zeros((blk.rows, blk.cols))
+    elif blk.mom_mode == MOM_LOWRANK:
+        st.L = np.zeros((blk.rows, blk.rank)) if L0 is None else np.array(L0, dtype=np.float64)
+        st.R = np.zeros((blk.rank, blk.cols))
+        assert st.L.shape == (blk.rows, blk.rank)
+    return st
+
+
+def block_step(W: np.ndarray, g: np.ndarray, st: BlockState, blk: Block, hp: HParams, t: int,
+               solver: str = "gd", keep: bool = False) -> np.ndarray:
+    """Advance one block by one step (t is 1-based).  Returns W_{t+1}; updates `st` in place."""
+    W = np.asarray(W, dtype=np.float64).reshape(blk.rows, blk.cols)
+    g = np.asarray(g, dtype=np.float64).reshape(blk.rows, blk.cols)
+    b1 = hp.beta1
+
+    # line 7 (or its group average)
+    st.v = second_moment(st.v, g, blk, hp.beta2)
+
+    if blk.mom_mode == MOM_NONE:
+        m_c = g
+    elif blk.mom_mode == MOM_FULL:
+        st.m = (1.0 - b1) * g + b1 * st.m                      # Eq. 4
+        m_c = st.m
+    elif blk.mom_mode == MOM_LOWRANK:
+        P_prev = st.L @ st.R
+        m_t = (1.0 - b1) * g + b1 * P_prev                     # line 4
+        if solver == "gd":
+            L, R = lowrank_refit_gd(m_t, st.L, st.R, hp.inner_iters, hp.inner_lr_scale)   # line 5
+        elif solver == "exact":
+            L, R = lowrank_refit_exact(m_t, blk.rank)
+        else:
+            raise ValueError(solver)
+        r_t = L @ R - m_t                                       # line 6
+        m_c = m_t - (b1 * r_t) / (1.0 - b1) if hp.correction else m_t   # line 8
+        st.L, st.R = L, R
+        if keep:
+            st.last = {"m_t": m_t, "r_t": r_t, "P_prev": P_prev, "P": L @ R}
+        if not (np.isfinite(L).all() and np.isfinite(R).all()):
+            raise FloatingPointError("low-rank factors are not finite")
+    else:
+        raise ValueError(blk.mom_mode)
+
+    v_el = _v_per_element(st.v, blk)
+    if hp.adam_debias:
+        m_hat = m_c / (1.0 - b1 ** t)
+        v_hat = v_el / (1.0 - hp.beta2 ** t)
+    else:
+        m_hat, v_hat = m_c, v_el
+    ratio = m_hat / (np.sqrt(v_hat) + hp.eps)
+    if math.isfinite(hp.clip):
+        ratio = np.clip(ratio, -hp.clip, hp.clip)
+    if keep:
+        st.last["m_c"] = m_c
+        st.last["ratio"] = ratio
+    # line 9, with x_t read as W_t
+    return W - (hp.lr * blk.lr_scale) * (ratio + blk.weight_decay * W)
+
+
+# ----------------------------------------------------------------------------------------------
+# A whole parameter set: blocks are independent of each other
+# ----------------------------------------------------------------------------------------------
+
+class AdaPMOracle:
+    def __init__(self, blocks: List[Block], hp: HParams, L0: Optional[Dict[int, np.ndarray]] = None,
+                 seed: int = 0):
+        self.blocks = list(blocks)
+        self.hp = hp
+        self.t = 0
+        self.states: List[BlockState] = []
+        for i, b in enumerate(self.blocks):
+            l0 = None
+            if b.mom_mode == MOM_LOWRANK:
+                l0 = L0[i] if (L0 is not None and i in L0) else init_L0(b.rows, b.rank, seed, i)
+            self.states.append(new_state(b, l0))
+
+    def step(self, params: List[np.ndarray], grads: List[np.ndarray], solver: str = "gd",
+             keep: bool = False) -> List[np.ndarray]:
+        self.t += 1
+        return [block_step(W, g, st, b, self.hp, self.t, solver, keep)
+                for W, g, st, b in zip(params, grads, self.states, self.blocks)]
+
+    def state_floats(self) -> int:
+        """Persistent optimizer-state size in scalars (momentum, factors, second moment)."""
+        n = 0
+        for b in self.blocks:
+            n += b.n_groups()
+            if b.mom_mode == MOM_FULL:
+                n += b.rows * b.cols
+            elif b.mom_mode == MOM_LOWRANK:
+                n += b.rank * (b.rows + b.cols)
+        return n

@@ -1,0 +1,380 @@
+"""Pins of the fp64 oracle against what the paper and the mathematics fix.
+
+None of these tests compares the oracle with itself: each uses a closed form, a
+special case that reduces to a library routine, an identity from the paper's
+proof of Theorem 2, or scalar brute force on tiny blocks.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import adapm_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+RNG = np.random.default_rng(1234)
+
+
+def _rand_block(rows, cols, **kw):
+    return O.Block(rows=rows, cols=cols, **kw)
+
+
+# ------------------------------------------------------------------------------------ schedule
+
+def test_inner_schedule_matches_closed_forms():
+    want = [float(l) for l in open(os.path.join(GOLD, "inner_schedule_K5.txt")) if l[0] not in "#\n"]
+    got = O.inner_schedule(5)
+    assert got[4] == 0.0                      # cos(pi) = -1 exactly: the 5th pass is a no-op
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-15)
+    s5 = math.sqrt(5.0)
+    np.testing.assert_allclose(got[:2], [0.5 * (1 + (1 + s5) / 4), 0.5 * (1 + (s5 - 1) / 4)], atol=1e-15)
+    assert all(a > b for a, b in zip(got, got[1:]))      # decreasing
+
+
+# ------------------------------------------------------------------------------------ P1
+
+def _plain_full_momentum_step(W, g, m, v, lr, b1, b2, eps, lam, clip):
+    """Eq. 4 + Algorithm 1 line 7 + line 9, written out on its own."""
+    m = b1 * m + (1 - b1) * g
+    v = b2 * v + (1 - b2) * g * g
+    u = m / (np.sqrt(v) + eps)
+    u = np.minimum(np.maximum(u, -clip), clip)
+    return W - lr * (u + lam * W), m, v
+
+
+def test_P1_all_full_equals_plain_routine():
+    rows, cols = 7, 5
+    blk = _rand_block(rows, cols, mom_mode=O.MOM_FULL, weight_decay=0.1)
+    hp = O.HParams(lr=3e-3, beta1=0.9, beta2=0.95)
+    st = O.new_state(blk)
+    W = RNG.standard_normal((rows, cols)); Wp = W.copy()
+    m = np.zeros_like(W); v = np.zeros_like(W)
+    for t in range(1, 8):
+        g = RNG.standard_normal((rows, cols)) * 1e-2
+        W = O.block_step(W, g, st, blk, hp, t)
+        Wp, m, v = _plain_full_momentum_step(Wp, g, m, v, 3e-3, 0.9, 0.95, 1e-8, 0.1, 1.0)
+        for a, b in ((W, Wp), (st.m, m), (st.v, v)):      # equal up to the order of two roundings
+            np.testing.assert_allclose(a, b, rtol=1e-15, atol=0)
+
+
+def test_P1_debiased_unclipped_full_momentum_is_textbook_adamw():
+    torch = pytest.importorskip("torch")
+    rows, cols = 6, 4
+    W0 = RNG.standard_normal((rows, cols))
+    p = torch.nn.Parameter(torch.tensor(W0, dtype=torch.float64))
+    opt = torch.optim.AdamW([p], lr=2e-3, betas=(0.9, 0.95), eps=1e-8, weight_decay=0.1)
+    blk = _rand_block(rows, cols, mom_mode=O.MOM_FULL, weight_decay=0.1)
+    hp = O.HParams(lr=2e-3, beta1=0.9, beta2=0.95, clip=math.inf, adam_debias=True)
+    st = O.new_state(blk)
+    W = W0.copy()
+    for t in range(1, 11):
+        g = RNG.standard_normal((rows, cols))
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        W = O.block_step(W, g, st, blk, hp, t)
+        np.testing.assert_allclose(W, p.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------------------------------ P2
+
+def test_P2_exact_solver_at_full_rank_is_full_momentum():
+    rows, cols = 6, 4
+    lr_blk = _rand_block(rows, cols, mom_mode=O.MOM_LOWRANK, rank=4, weight_decay=0.1)
+    fm_blk = _rand_block(rows, cols, mom_mode=O.MOM_FULL, weight_decay=0.1)
+    hp = O.HParams()
+    s1, s2 = O.new_state(lr_blk), O.new_state(fm_blk)
+    W1 = RNG.standard_normal((rows, cols)); W2 = W1.copy()
+    for t in range(1, 13):
+        g = RNG.standard_normal((rows, cols)) * 1e-3
+        W1 = O.block_step(W1, g, s1, lr_blk, hp, t, solver="exact", keep=True)
+        W2 = O.block_step(W2, g, s2, fm_blk, hp, t)
+        assert np.abs(s1.last["r_t"]).max() < 1e-15
+        np.testing.assert_allclose(s1.last["m_c"], s2.m, rtol=0, atol=1e-15)
+        np.testing.assert_allclose(W1, W2, rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------------------------------ P3
+
+def test_P3_constant_gradient_closed_forms_full_none_and_v():
+    rows, cols, b1, b2, eps, lr = 4, 6, 0.9, 0.95, 1e-8, 1e-3
+    g = RNG.standard_normal((rows, cols)) * 1e-3
+    hp = O.HParams(lr=lr, beta1=b1, beta2=b2, eps=eps)
+    full = _rand_block(rows, cols, mom_mode=O.MOM_FULL)
+    none = _rand_block(rows, cols, mom_mode=O.MOM_NONE, lr_scale=0.75)
+    bm = _rand_block(rows, cols, mom_mode=O.MOM_NONE, v_mode=O.V_BLOCKMEAN, v_group_rows=2)
+    sf, sn, sb = O.new_state(full), O.new_state(none), O.new_state(bm)
+    Wf = np.zeros((rows, cols)); Wn = Wf.copy(); Wb = Wf.copy()
+    acc_f = np.zeros_like(Wf); acc_n = np.zeros_like(Wf); acc_b = np.zeros_like(Wf)
+    for t in range(1, 16):
+        Wf = O.block_step(Wf, g, sf, full, hp, t)
+        Wn = O.block_step(Wn, g, sn, none, hp, t)
+        Wb = O.block_step(Wb, g, sb, bm, hp, t)
+        np.testing.assert_allclose(sf.m, (1 - b1 ** t) * g, rtol=1e-13)
+        np.testing.assert_allclose(sf.v, (1 - b2 ** t) * g * g, rtol=1e-13)
+        mean_sq = (g * g).reshape(2, 2 * cols).mean(axis=1)
+        np.testing.assert_allclose(sb.v, (1 - b2 ** t) * mean_sq, rtol=1e-13)
+        den = math.sqrt(1 - b2 ** t) * np.abs(g) + eps
+        acc_f += np.clip((1 - b1 ** t) * g / den, -1, 1)
+        acc_n += np.clip(g / den, -1, 1)
+        den_b = np.sqrt((1 - b2 ** t) * np.repeat(mean_sq, 2))[:, None] + eps
+        acc_b += np.clip(g / den_b, -1, 1)
+        np.testing.assert_allclose(Wf, -lr * acc_f, rtol=1e-12, atol=1e-18)     # lambda = 0
+        np.testing.assert_allclose(Wn, -lr * 0.75 * acc_n, rtol=1e-12, atol=1e-18)
+        np.testing.assert_allclose(Wb, -lr * acc_b, rtol=1e-12, atol=1e-18)
+
+
+def test_P3_constant_gradient_lowrank_exact_closed_form():
+    rows, cols, r, b1 = 7, 5, 2, 0.9
+    U, _ = np.linalg.qr(RNG.standard_normal((rows, cols)))
+    Vt, _ = np.linalg.qr(RNG.standard_normal((cols, cols)))
+    sig = np.array([5.0, 3.0, 1.0, 0.5, 0.25]) * 1e-3
+    g = (U * sig) @ Vt.T
+    head = (U[:, :r] * sig[:r]) @ Vt[:, :r].T
+    tail = g - head
+    blk = _rand_block(rows, cols, mom_mode=O.MOM_LOWRANK, rank=r)
+    hp = O.HParams(beta1=b1)
+    st = O.new_state(blk)
+    W = np.zeros((rows, cols))
+    for t in range(1, 15):
+        W = O.block_step(W, g, st, blk, hp, t, solver="exact", keep=True)
+        np.testing.assert_allclose(st.last["P"], (1 - b1 ** t) * head, rtol=0, atol=1e-15)
+        np.testing.assert_allclose(st.last["m_t"], (1 - b1 ** t) * head + (1 - b1) * tail, atol=1e-15)
+        np.testing.assert_allclose(st.last["r_t"], -(1 - b1) * tail, atol=1e-15)
+        np.testing.assert_allclose(st.last["m_c"], (1 - b1 ** t) * head + tail, atol=1e-14)
+    # rank(g) <= r: the corrected momentum is the full momentum
+    g2 = head
+    st = O.new_state(blk)
+    for t in range(1, 8):
+        O.block_step(W, g2, st, blk, hp, t, solver="exact", keep=True)
+        np.testing.assert_allclose(st.last["m_c"], (1 - b1 ** t) * g2, atol=1e-15)
+
+
+# ------------------------------------------------------------------------------------ P4
+
+@pytest.mark.parametrize("solver", ["gd", "exact"])
+def test_P4_proof_identity_along_a_trajectory(solver):
+    """m_t - m^f_t = sum_{i=1}^{t-1} beta1^i r_{t-i} and m^c_t = g_t + c (P_{t-1} - P_t), for any solver
+    (proof of Theorem 2, first display: m_t - m^f_t = beta1 (m_{t-1} - m^f_{t-1}) + beta1 r_{t-1})."""
+    rows, cols, r, b1 = 24, 16, 3, 0.9
+    blk = _rand_block(rows, cols, mom_mode=O.MOM_LOWRANK, rank=r)
+    hp = O.HParams(beta1=b1)
+    st = O.new_state(blk, O.init_L0(rows, r, 0, 0))
+    W = RNG.standard_normal((rows, cols)) * 0.02
+    mf = np.zeros((rows, cols))
+    residuals = []
+    c = b1 / (1 - b1)
+    for t in range(1, 21):
+        g = RNG.standard_normal((rows, cols)) * 1e-3 + 2e-3 * np.outer(np.sin(np.arange(rows)), np.cos(np.arange(cols)))
+        W = O.block_step(W, g, st, blk, hp, t, solver=solver, keep=True)
+        mf = (1 - b1) * g + b1 * mf
+        want = sum(b1 ** i * residuals[t - 1 - i] for i in range(1, t))
+        scale = np.abs(mf).max()
+        assert np.abs(st.last["m_t"] - mf - want).max() < 1e-13 * scale + 1e-18
+        assert np.abs(st.last["m_c"] - (g + c * (st.last["P_prev"] - st.last["P"]))).max() < 1e-12 * scale
+        residuals.append(st.last["r_t"])
+
+
+def test_P4_constant_residual_gives_theorem2_gap():
+    """If r_t = r for all t >= 1 then m^c_t - m^f_t = -beta1^t r / (1 - beta1)  (r_0 = 0)."""
+    b1, T = 0.9, 12
+    r = 0.37
+    # scalar recursion of the proof: d_t = beta1 d_{t-1} + beta1 r_{t-1}, d_0 = 0, r_0 = 0
+    d = 0.0
+    prev_r = 0.0
+    for t in range(1, T + 1):
+        d = b1 * d + b1 * prev_r
+        prev_r = r
+        gap = d - b1 * r / (1 - b1)
+        assert abs(gap - (-(b1 ** t) * r / (1 - b1))) < 1e-14
+
+
+# ------------------------------------------------------------------------------------ P5
+
+def _alg2_scalar_rank1(M, l, rho, K):
+    """Algorithm 2 for rank 1 with explicit index loops (no matrix products)."""
+    m, n = len(l), len(rho)
+    l = list(l); rho = list(rho)
+    for k in range(1, K + 1):
+        eta = 0.5 * (1 + math.cos(math.pi * k / K))
+        E = [[l[i] * rho[j] - M[i][j] for j in range(n)] for i in range(m)]
+        dl = [sum(E[i][j] * rho[j] for j in range(n)) for i in range(m)]
+        dr = [sum(l[i] * E[i][j] for i in range(m)) for j in range(n)]
+        l = [l[i] - eta * dl[i] for i in range(m)]
+        rho = [rho[j] - eta * dr[j] for j in range(n)]
+    return l, rho
+
+
+@pytest.mark.parametrize("shape", [(2, 2), (3, 2), (2, 3)])
+def test_P5_alg2_brute_force_rank1(shape):
+    m, n = shape
+    M = RNG.standard_normal((m, n))
+    l0 = RNG.standard_normal(m) * 0.5
+    r0 = RNG.standard_normal(n) * 0.5
+    L, R = O.lowrank_refit_gd(M, l0[:, None], r0[None, :], 5)
+    l, rho = _alg2_scalar_rank1(M.tolist(), l0.tolist(), r0.tolist(), 5)
+    np.testing.assert_allclose(L[:, 0], l, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(R[0, :], rho, rtol=1e-13, atol=1e-15)
+
+
+def test_P5_alg2_derivatives_by_finite_differences():
+    """The printed derivatives are those of l = 0.5 ||L R - m_t||_F^2 (no factor 2)."""
+    m, n, r = 4, 3, 2
+    M = RNG.standard_normal((m, n)); L = RNG.standard_normal((m, r)); R = RNG.standard_normal((r, n))
+    loss = lambda L_, R_: 0.5 * np.sum((L_ @ R_ - M) ** 2)
+    h = 1e-6
+    # one pass with K=2 has eta_1 = 0.5, eta_2 = 0: the move is -0.5 * derivative
+    L1, R1 = O.lowrank_refit_gd(M, L, R, 2)
+    dL = (L - L1) / 0.5
+    dR = (R - R1) / 0.5
+    for i in range(m):
+        for k in range(r):
+            Lp = L.copy(); Lp[i, k] += h; Lm = L.copy(); Lm[i, k] -= h
+            assert abs((loss(Lp, R) - loss(Lm, R)) / (2 * h) - dL[i, k]) < 1e-6
+    for k in range(r):
+        for j in range(n):
+            Rp = R.copy(); Rp[k, j] += h; Rm = R.copy(); Rm[k, j] -= h
+            assert abs((loss(L, Rp) - loss(L, Rm)) / (2 * h) - dR[k, j]) < 1e-6
+
+
+def test_P5_exact_solver_vs_2x2_closed_form_and_power_iteration():
+    a, b, c, d = RNG.standard_normal(4)
+    M = np.array([[a, b], [c, d]])
+    S1 = a * a + b * b + c * c + d * d
+    S2 = math.sqrt((a * a + b * b - c * c - d * d) ** 2 + 4 * (a * c + b * d) ** 2)
+    s_small = math.sqrt((S1 - S2) / 2)
+    L, R = O.lowrank_refit_exact(M, 1)
+    assert abs(np.linalg.norm(L @ R - M) - s_small) < 1e-13
+    # power iteration for the leading pair on a 5x4 matrix
+    A = RNG.standard_normal((5, 4))
+    x = np.ones(4)
+    for _ in range(2000):
+        x = A.T @ (A @ x); x /= np.linalg.norm(x)
+    P_pow = np.outer(A @ x, x)
+    L, R = O.lowrank_refit_exact(A, 1)
+    np.testing.assert_allclose(L @ R, P_pow, atol=1e-10)
+
+
+def test_alg2_descends_and_tracks_a_low_rank_target():
+    rows, cols, r = 40, 30, 3
+    M = (RNG.standard_normal((rows, r)) @ RNG.standard_normal((r, cols))) * 0.005   # curvature eta*||R R^T|| << 1
+    L = O.init_L0(rows, r, 0, 7); R = np.zeros((r, cols))
+    prev = np.linalg.norm(L @ R - M)
+    for _ in range(300):
+        L, R = O.lowrank_refit_gd(M, L, R, 5)
+        cur = np.linalg.norm(L @ R - M)
+        assert cur <= prev * (1 + 1e-12)
+        prev = cur
+    assert prev < 1e-3 * np.linalg.norm(M)
+
+
+def test_init_L0_is_orthonormal_and_fp32():
+    L0 = O.init_L0(200, 12, 3, 5)
+    assert np.array_equal(L0, L0.astype(np.float32).astype(np.float64))
+    np.testing.assert_allclose(L0.T @ L0, np.eye(12), atol=5e-7)
+    assert not np.array_equal(L0, O.init_L0(200, 12, 3, 6))
+    assert np.array_equal(L0, O.init_L0(200, 12, 3, 5))
+
+
+# ------------------------------------------------------------------------------------ P6
+
+def test_P6_blockmean_is_group_average_of_elementwise_v():
+    rows, cols = 12, 5
+    el = _rand_block(rows, cols, mom_mode=O.MOM_NONE)
+    for gr in (0, 1, 3, 12):
+        bm = _rand_block(rows, cols, mom_mode=O.MOM_NONE, v_mode=O.V_BLOCKMEAN, v_group_rows=gr)
+        se, sb = O.new_state(el), O.new_state(bm)
+        hp = O.HParams()
+        W = np.zeros((rows, cols))
+        for t in range(1, 9):
+            g = RNG.standard_normal((rows, cols))
+            O.block_step(W, g, se, el, hp, t)
+            O.block_step(W, g, sb, bm, hp, t)
+            k = rows if gr == 0 else gr
+            np.testing.assert_allclose(sb.v, se.v.reshape(rows // k, k * cols).mean(axis=1), rtol=1e-13)
+
+
+# ------------------------------------------------------------------------------------ P7
+
+def test_P7_no_refit_or_zero_factors_reduce_to_no_momentum():
+    rows, cols, r = 9, 6, 2
+    none = _rand_block(rows, cols, mom_mode=O.MOM_NONE, weight_decay=0.1)
+    lowr = _rand_block(rows, cols, mom_mode=O.MOM_LOWRANK, rank=r, weight_decay=0.1)
+    for K, L0 in ((0, O.init_L0(rows, r, 0, 0)), (5, np.zeros((rows, r)))):
+        hp = O.HParams(inner_iters=K)
+        sn, sl = O.new_state(none), O.new_state(lowr, L0)
+        Wn = RNG.standard_normal((rows, cols)) * 0.02; Wl = Wn.copy()
+        for t in range(1, 7):
+            g = RNG.standard_normal((rows, cols)) * 1e-3
+            Wn = O.block_step(Wn, g, sn, none, hp, t)
+            Wl = O.block_step(Wl, g, sl, lowr, hp, t)
+            np.testing.assert_allclose(Wl, Wn, rtol=0, atol=1e-15)
+            assert not sl.R.any()
+
+
+def test_P7_last_pass_is_a_noop():
+    M = RNG.standard_normal((6, 5)) * 0.1
+    L = O.init_L0(6, 2, 0, 1); R = RNG.standard_normal((2, 5)) * 0.1
+    L5, R5 = O.lowrank_refit_gd(M, L, R, 5)
+    # four passes by hand with the K=5 step sizes
+    La, Ra = L.copy(), R.copy()
+    for k in (1, 2, 3, 4):
+        eta = 0.5 * (1 + math.cos(math.pi * k / 5))
+        E = La @ Ra - M
+        La, Ra = La - eta * (E @ Ra.T), Ra - eta * (La.T @ E)
+    assert np.array_equal(L5, La) and np.array_equal(R5, Ra)
+
+
+# ------------------------------------------------------------------------------------ P8
+
+def test_P8_zero_padded_rank_changes_nothing():
+    rows, cols, r, pad = 10, 8, 3, 5
+    M = RNG.standard_normal((rows, cols)) * 0.05
+    L = O.init_L0(rows, r, 0, 2); R = RNG.standard_normal((r, cols)) * 0.05
+    Lp = np.hstack([L, np.zeros((rows, pad - r))]); Rp = np.vstack([R, np.zeros((pad - r, cols))])
+    L1, R1 = O.lowrank_refit_gd(M, L, R, 5)
+    L2, R2 = O.lowrank_refit_gd(M, Lp, Rp, 5)
+    np.testing.assert_allclose(L2[:, :r], L1, rtol=0, atol=1e-16)
+    np.testing.assert_allclose(R2[:r], R1, rtol=0, atol=1e-16)
+    assert not L2[:, r:].any() and not R2[r:].any()
+
+
+# ------------------------------------------------------------------------------------ P10
+
+def test_P10_blocks_are_independent():
+    blocks = [
+        O.Block(6, 4, O.MOM_FULL, weight_decay=0.1),
+        O.Block(8, 6, O.MOM_LOWRANK, rank=2, weight_decay=0.1, v_mode=O.V_BLOCKMEAN, v_group_rows=2),
+        O.Block(5, 3, O.MOM_NONE, lr_scale=0.75),
+    ]
+    L0 = {1: O.init_L0(8, 2, 0, 99)}
+    a = O.AdaPMOracle(blocks, O.HParams(), L0=L0)
+    b = O.AdaPMOracle([blocks[1]], O.HParams(), L0={0: L0[1]})
+    Wa = [RNG.standard_normal((x.rows, x.cols)) * 0.02 for x in blocks]
+    Wb = [Wa[1].copy()]
+    for _ in range(6):
+        gs = [RNG.standard_normal((x.rows, x.cols)) * 1e-3 for x in blocks]
+        Wa = a.step(Wa, gs)
+        Wb = b.step(Wb, [gs[1]])
+    assert np.array_equal(Wa[1], Wb[0])
+    assert np.array_equal(a.states[1].L, b.states[0].L)
+
+
+# ------------------------------------------------------------------------------------ weight decay / clip
+
+def test_weight_decay_is_decoupled_and_clip_is_elementwise():
+    blk = _rand_block(1, 3, mom_mode=O.MOM_NONE, weight_decay=0.5)
+    hp = O.HParams(lr=0.1, beta2=0.0, eps=0.0)       # v = g^2 -> ratio = sign(g)
+    st = O.new_state(blk)
+    W = np.array([[2.0, -4.0, 8.0]])
+    g = np.array([[3.0, -0.5, 0.0]])
+    hp.eps = 1e-8
+    W1 = O.block_step(W, g, st, blk, hp, 1)
+    want = W - 0.1 * (np.array([[1.0, -1.0, 0.0]]) + 0.5 * W)
+    np.testing.assert_allclose(W1, want, rtol=1e-7)
+    # the clamp acts per element: one large ratio does not shrink the others
+    blk2 = _rand_block(1, 2, mom_mode=O.MOM_NONE)
+    st2 = O.new_state(blk2); st2.v = np.array([[1.0, 1.0]])
+    hp2 = O.HParams(lr=1.0, beta2=1.0, eps=0.0)
+    W2 = O.block_step(np.zeros((1, 2)), np.array([[10.0, 0.25]]), st2, blk2, hp2, 1)
+    np.testing.assert_allclose(W2, [[-1.0, -0.25]], rtol=1e-15)
