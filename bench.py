@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the AdaPM optimizer step (one step = one adapm_step over every block of a parameter set).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload gpt2_1p5b] [--v-mode blockmean]
+  python bench.py --impl reference ...      # times the fp64 CPU oracle instead (a deliberately slow baseline)
+
+Prints ONE JSON line (rank 0).  `value` = optimizer steps per second with every input resident in HBM,
+timed with CUDA events over exactly K steps; `e2e` = the same with the step's gradients copied from pinned
+host memory and the updated parameters copied back inside the timed region.  With N > 1 the N ranks run
+independent replicas of the same set (the step has no cross-GPU exchange); value = all ranks' steps / max time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "adapm_optimizer_steps_per_sec"
+UNIT = "steps/s"
+SM_COUNT, FMA_LANES = 148, 128
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload
+# (profiles/ holds the captures these come from); None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+# ------------------------------------------------------------------------------------------------ oracle arm
+
+def _class_key(b):
+    return (b.mom_mode, b.rows, b.cols, b.rank, b.v_mode, b.v_group_rows)
+
+
+def oracle_step_estimate(w, blocks, max_rows: int = 4096, seed: int = 0):
+    """Time one oracle step on one block of every class and scale by the class sizes.
+
+    Returns (estimated seconds for a full step, description of the sample).  Blocks with more than
+    `max_rows` rows and no low-rank factors are timed on their first `max_rows` rows and scaled.
+    """
+    from oracle import adapm_oracle as O
+    import workloads as WL
+    classes = {}
+    for i, b in enumerate(blocks):
+        classes.setdefault(_class_key(b), []).append(i)
+    hp = O.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
+    rng = np.random.default_rng(seed)
+    total, sampled_elems = 0.0, 0
+    for key, ids in classes.items():
+        b = blocks[ids[0]]
+        rows = b.rows
+        scale = 1.0
+        if b.mom_mode != O.MOM_LOWRANK and rows > max_rows:
+            gr = max(b.v_group_rows, 1)
+            rows = max_rows // gr * gr
+            scale = b.rows / rows
+        ob = O.Block(rows, b.cols, b.mom_mode, b.rank, b.v_mode, b.v_group_rows, b.lr_scale, b.weight_decay)
+        L0 = O.init_L0(rows, b.rank, 0, ids[0]) if b.mom_mode == O.MOM_LOWRANK else None
+        st = O.new_state(ob, L0)
+        W = rng.standard_normal((rows, b.cols)) * 0.02
+        g, _ = WL.to_grad_dtype((rng.standard_normal((rows, b.cols)) * 1e-3).astype(np.float32), w.grad_dtype)
+        g = g.astype(np.float64)
+        t0 = time.perf_counter()
+        O.block_step(W, g, st, ob, hp, 1)
+        dt = time.perf_counter() - t0
+        total += dt * scale * len(ids)
+        sampled_elems += rows * b.cols
+    desc = (f"one block of each of {len(classes)} block classes (non-low-rank blocks capped at {max_rows} rows), "
+            f"{sampled_elems} of {sum(b.rows * b.cols for b in blocks)} elements, one step each, "
+            f"scaled by class size")
+    return total, desc
+
+
+def _blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return 1
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import workloads as WL
+    from oracle import planner_oracle as P
+    w = WL.get_workload(args.workload)
+    blocks = P.plan(w.tensors, w.weight_decay, w.rank_pct, args.v_mode == "blockmean")
+    times, desc = [], ""
+    for i in range(args.warmup + args.steps):
+        t, desc = oracle_step_estimate(w, blocks, seed=i)
+        if i >= args.warmup:
+            times.append(t)
+    sec = float(np.mean(times))
+    val = 1.0 / sec
+    cores = _blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "params": w.numel, "v_mode": args.v_mode, "grad_dtype": w.grad_dtype},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ GPU arm
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def kernel_algorithmic_work(kind: str, blocks, gsz: int, k_eff: int):
+    """(bound, amount, unit) of one launch of `kind`: bytes for HBM-bound kernels, flops for the others."""
+    import paper_2510_09103_b200 as A
+    nb = lambda b: b.rows * b.cols
+    groups = lambda b: nb(b) if b.v_mode == A.V_ELEMENT else (1 if b.v_group_rows == 0 else b.rows // b.v_group_rows)
+    lowr = [b for b in blocks if b.mom_mode == A.MOM_LOWRANK]
+    if kind == "stream_update":
+        tot = 0
+        for b in blocks:
+            if b.mom_mode == A.MOM_LOWRANK:
+                continue
+            tot += nb(b) * (gsz + 8 + (8 if b.mom_mode == A.MOM_FULL else 0)) + groups(b) * 8
+        return "hbm", tot, "bytes"
+    if kind in ("apply_simt", "tc_apply"):
+        # g + W in, W out, plus the factors once; flops of the rank-2r product reported separately
+        tot = sum(nb(b) * (gsz + 8) + groups(b) * (8 if b.v_mode == A.V_ELEMENT else 4)
+                  + 2 * 4 * b.rank * (b.rows + b.cols) for b in lowr)
+        return "hbm", tot, "bytes"
+    if kind == "gemm_simt":
+        # averaged over the 4 GEMM launches of one refit pass: (4 m n r + 8 r^2 (m + n)) / 4
+        fl = sum(4.0 * nb(b) * b.rank + 8.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr) / 4.0
+        return "alu", fl, "flops"
+    if kind == "tc_panel":
+        fl = sum(4.0 * nb(b) * b.rank for b in lowr)
+        return "tensor", fl, "flops"
+    if kind in ("reduce_partial",):
+        return "hbm", sum(nb(b) * gsz for b in lowr), "bytes"
+    return "hbm", 0, "bytes"
+
+
+def run_gpu(args) -> None:
+    import torch
+    import workloads as WL
+    import paper_2510_09103_b200 as A
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the optimizer step has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    w = WL.get_workload(args.workload)
+    blockmean = args.v_mode == "blockmean"
+    blocks, total = A.adapm_plan_default(w.tensors, w.rank_pct, w.rank_override,
+                                         A.V_BLOCKMEAN if blockmean else A.V_ELEMENT, w.weight_decay)
+    gd = A.GRAD_BF16 if w.grad_dtype == "bf16" else A.GRAD_F32
+    gsz = 2 if w.grad_dtype == "bf16" else 4
+    path = {"auto": A.PATH_AUTO, "simt": A.PATH_SIMT, "tensor": A.PATH_TENSOR}[args.path]
+    hp = A.hparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, grad_dtype=gd, lowrank_path=path)
+    ctx = A.adapm_create(blocks, hp)
+
+    # synthetic inputs: parameters N(0, 0.02^2) drawn on the device; gradients tiled from a seeded host pool
+    gen = torch.Generator(device=dev); gen.manual_seed(1)
+    params = torch.empty(total, dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=gen)
+    pool = WL.GradPool(w, pool_elems=1 << 24)
+    raw = pool.raw.view(np.int16) if w.grad_dtype == "bf16" else pool.raw
+    tdt = torch.int16 if w.grad_dtype == "bf16" else torch.float32
+    pool_t = torch.from_numpy(raw)
+    grads_host = torch.empty(total, dtype=tdt, pin_memory=True)
+    reps = -(-total // pool_t.numel())
+    grads_host.copy_(pool_t.repeat(reps)[:total])
+    grads = torch.empty(total, dtype=torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32, device=dev)
+    grads.view(tdt).copy_(grads_host)
+    state = torch.zeros(ctx.adapm_state_bytes() // 4, dtype=torch.float32, device=dev)
+    work = torch.zeros(max(ctx.adapm_workspace_bytes() // 4, 64), dtype=torch.float32, device=dev)
+    ctx.adapm_set_workspace(work)
+    ctx.adapm_state_init(state)
+    torch.cuda.synchronize()
+
+    t = 0
+
+    def do_steps(n):
+        nonlocal t
+        for _ in range(n):
+            t += 1
+            ctx.adapm_step(params, grads, state, t)
+
+    # ---- device-resident timing ----
+    do_steps(args.warmup)
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    do_steps(args.steps)
+    e1.record()
+    barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop() if sampler else None
+    status = ctx.adapm_get_status()
+    if status != 0:
+        raise SystemExit(f"device status word {status}: a bounded wait expired; numbers are invalid")
+    ms_step = ms_total / args.steps
+    value = world * args.steps / (ms_total * 1e-3)
+
+    # ---- per-kernel durations (separate profiled pass; CUDA events on the launching stream) ----
+    per_kind = {}
+    ctx.adapm_set_profiling(True)
+    for _ in range(args.steps):
+        do_steps(1)
+        for kind, ms in ctx.adapm_get_launch_times():
+            d = per_kind.setdefault(kind, [0, 0.0])
+            d[0] += 1; d[1] += ms
+    ctx.adapm_set_profiling(False)
+    tot_ms = sum(v[1] for v in per_kind.values()) or 1.0
+    kernels = {k: {"launches_per_step": v[0] / args.steps, "ms_per_step": v[1] / args.steps, "share": v[1] / tot_ms}
+               for k, v in per_kind.items()}
+
+    # ---- end to end: host gradients in, updated parameters out, inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        params_host = torch.empty(total, dtype=torch.float32, pin_memory=True)
+        for _ in range(2):
+            grads.view(tdt).copy_(grads_host, non_blocking=True); do_steps(1); params_host.copy_(params, non_blocking=True)
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            grads.view(tdt).copy_(grads_host, non_blocking=True)
+            do_steps(1)
+            params_host.copy_(params, non_blocking=True)
+        e1.record()
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1))
+        e2e = {"value": world * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": total * gsz,
+               "d2h_bytes_per_step": total * 4, "ms_per_step": ms_e2e / args.steps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    k_eff = 4
+    step_bytes = ctx.adapm_step_bytes()
+    dom = max(kernels, key=lambda k: kernels[k]["share"]) if kernels else "stream_update"
+
+    def roofline_of(kind):
+        if kind not in kernels or kernels[kind]["launches_per_step"] == 0:
+            return None
+        bound, amount, _ = kernel_algorithmic_work(kind, blocks, gsz, k_eff)
+        sec = kernels[kind]["ms_per_step"] / kernels[kind]["launches_per_step"] * 1e-3
+        if bound == "hbm":
+            ach, peak, unit = amount / sec / 1e9, peaks["hbm_gbs"], "GB/s"
+        elif bound == "tensor":
+            ach, peak, unit = amount / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
+        else:
+            ach, peak, unit = amount / sec / 1e12, SM_COUNT * FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12, "TFLOP/s"
+        return {"kernel": kind, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get(f"{kind}:{w.name}:{args.v_mode}"), "peak_source": peaks["source"],
+                "per_launch_ms": sec * 1e3, "algorithmic_per_launch": amount}
+
+    cpu_s, cpu_desc = oracle_step_estimate(w, blocks)
+    sb = ctx.adapm_state_breakdown()
+    state_bytes = sum(sb.values())
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "params": w.numel, "blocks": len(blocks), "v_mode": args.v_mode,
+                   "grad_dtype": w.grad_dtype, "state_dtype": "f32", "lowrank_path": args.path,
+                   "lowrank_kernels": "tensor" if any(k.startswith("tc_") for k in kernels) else "simt",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (no flush between steps)"},
+        "params_per_s": value * w.numel,
+        "step_bytes": step_bytes, "step_gbs": step_bytes / (ms_step * 1e-3) / 1e9,
+        "step_hbm_frac_of_measured": step_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "step_hbm_frac_of_8tbs": step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0,
+        "step_contraction_tflops": ctx.adapm_step_flops() / (ms_step * 1e-3) / 1e12,
+        "state_bytes": state_bytes, "state_breakdown": sb, "adamw_state_bytes": 8 * w.numel,
+        "state_saving_vs_adamw": 1.0 - state_bytes / (8.0 * w.numel),
+        "gpu_launches": ctx.adapm_launch_count() * args.steps,
+        "kernels": kernels,
+        "roofline": roofline_of(dom),
+        "roofline_stream_update": roofline_of("stream_update"),
+        "clocks": clocks,
+        "e2e": e2e,
+        "cpu_baseline": {"value": 1.0 / cpu_s, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+                         "sample": cpu_desc, "est_s_per_step": cpu_s},
+    }
+    print(json.dumps(line))
+    ctx.adapm_destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="gpt2_1p5b")
+    ap.add_argument("--v-mode", default="blockmean", choices=["blockmean", "element"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

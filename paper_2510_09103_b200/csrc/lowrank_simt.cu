@@ -1,0 +1,257 @@
+// CUDA-core (FFMA) kernels of the low-rank path: a batched strided GEMM that carries every product
+// of Algorithm 2, the fused "apply" kernel that rebuilds m^c = cg g + c0 L0 R0 - c1 L R tile by tile
+// and writes the parameters, and the L_0 initialiser.  This path is exact fp32 and handles every
+// shape and gradient dtype; the tensor-core path replaces it where its layout rules are met.
+#include "adapm_internal.h"
+#include "device_math.cuh"
+
+namespace adapm {
+
+namespace {
+
+constexpr int TM = 64, TN = 64, TK = 16;
+
+template <bool BF16G>
+__device__ __forceinline__ float load_operand(const void* base, bool is_grad, int64_t idx) {
+  if (is_grad) {
+    if (BF16G) return bf16_bits_to_float(static_cast<const uint16_t*>(base)[idx]);
+    return static_cast<const float*>(base)[idx];
+  }
+  return static_cast<const float*>(base)[idx];
+}
+
+// acc[4][4] += X(i0.., k) Y(k, j0..) over k in [0, K); thread (ty, tx) owns rows ty*4.., cols tx*4..
+template <bool BF16G>
+__device__ __forceinline__ void tile_mainloop(float (&acc)[4][4], const void* X, bool x_grad, int64_t sxi,
+                                              int64_t sxk, const void* Y, bool y_grad, int64_t syk, int64_t syj,
+                                              int M, int N, int K, int i0, int j0, float (*Xs)[TM + 4],
+                                              float (*Ys)[TN + 4]) {
+  const int t = threadIdx.x;
+  const int ty = t >> 4, tx = t & 15;
+  for (int k0 = 0; k0 < K; k0 += TK) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      int ii, kk;
+      if (sxk == 1) { kk = t & 15; ii = (t >> 4) + 16 * q; } else { ii = t & 63; kk = (t >> 6) + 4 * q; }
+      const int i = i0 + ii, k = k0 + kk;
+      Xs[kk][ii] = (i < M && k < K) ? load_operand<BF16G>(X, x_grad, (int64_t)i * sxi + (int64_t)k * sxk) : 0.f;
+      int jj, kj;
+      if (syj == 1) { jj = t & 63; kj = (t >> 6) + 4 * q; } else { kj = t & 15; jj = (t >> 4) + 16 * q; }
+      const int j = j0 + jj, k2 = k0 + kj;
+      Ys[kj][jj] = (j < N && k2 < K) ? load_operand<BF16G>(Y, y_grad, (int64_t)k2 * syk + (int64_t)j * syj) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < TK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&Xs[kk][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Ys[kk][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w};
+      const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], bv[c], acc[r][c]);
+    }
+    __syncthreads();
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ const T& find_by_first_tile(const T* tab, int n, int64_t me) {
+  int lo = 0, hi = n - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (tab[mid].first_tile <= me) lo = mid; else hi = mid - 1;
+  }
+  return tab[lo];
+}
+
+template <bool BF16G>
+__global__ void __launch_bounds__(256) gemm_kernel(const GemmProb* __restrict__ tab, int n_prob, Bases b) {
+  __shared__ __align__(16) float Xs[TK][TM + 4];
+  __shared__ __align__(16) float Ys[TK][TN + 4];
+  __shared__ GemmProb sP;
+  if (threadIdx.x == 0) sP = find_by_first_tile(tab, n_prob, (int64_t)blockIdx.x);
+  __syncthreads();
+  const GemmProb& P = sP;
+  const int64_t tile = (int64_t)blockIdx.x - P.first_tile;
+  const int i0 = (int)(tile / P.tiles_n) * TM, j0 = (int)(tile % P.tiles_n) * TN;
+
+  const size_t xsz = (P.x_base == BASE_GRADS && BF16G) ? 2 : 4, ysz = (P.y_base == BASE_GRADS && BF16G) ? 2 : 4;
+  const void* X = static_cast<const char*>(b.p[P.x_base]) + (size_t)P.x_off * xsz;
+  const void* Y = static_cast<const char*>(b.p[P.y_base]) + (size_t)P.y_off * ysz;
+  float acc[4][4] = {};
+  tile_mainloop<BF16G>(acc, X, P.x_base == BASE_GRADS, P.sxi, P.sxk, Y, P.y_base == BASE_GRADS, P.syk, P.syj, P.M,
+                       P.N, P.K, i0, j0, Xs, Ys);
+
+  float* C = static_cast<float*>(b.p[P.c_base]) + P.c_off;
+  const float* Z1 = P.z1_base >= 0 ? static_cast<const float*>(b.p[P.z1_base]) + P.z1_off : nullptr;
+  const float* Z2 = P.z2_base >= 0 ? static_cast<const float*>(b.p[P.z2_base]) + P.z2_off : nullptr;
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = i0 + ty * 4 + r;
+    if (i >= P.M) continue;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int j = j0 + tx * 4 + c;
+      if (j >= P.N) continue;
+      const int64_t o = (int64_t)i * P.ldc + j;
+      float x = P.alpha * acc[r][c];
+      if (P.beta != 0.f) x += P.beta * C[o];
+      if (Z1) x += P.c1 * Z1[o];
+      if (Z2) x += P.c2 * Z2[o];
+      C[o] = x;
+    }
+  }
+}
+
+template <bool BF16G>
+__global__ void __launch_bounds__(256) apply_simt_kernel(const ApplyBlk* __restrict__ tab, int n_blk, Bases b,
+                                                         StepScalars sc) {
+  __shared__ __align__(16) float Xs[TK][TM + 4];
+  __shared__ __align__(16) float Ys[TK][TN + 4];
+  __shared__ ApplyBlk sA;
+  if (threadIdx.x == 0) sA = find_by_first_tile(tab, n_blk, (int64_t)blockIdx.x);
+  __syncthreads();
+  const ApplyBlk& A = sA;
+  const int64_t tile = (int64_t)blockIdx.x - A.first_tile;
+  const int i0 = (int)(tile / A.tiles_n) * TM, j0 = (int)(tile % A.tiles_n) * TN;
+  const int m = A.rows, n = A.cols, r = A.rank;
+
+  float* state = static_cast<float*>(b.p[BASE_STATE]);
+  const float* L0 = state + A.l0_off;
+  const float* R0 = state + A.r0_off;
+  const float* L1 = static_cast<const float*>(b.p[A.l1_base]) + A.l1_off;
+  const float* R1 = static_cast<const float*>(b.p[A.l1_base]) + A.r1_off;
+
+  float p0[4][4] = {}, p1[4][4] = {};
+  tile_mainloop<BF16G>(p0, L0, false, r, 1, R0, false, n, 1, m, n, r, i0, j0, Xs, Ys);   // P_{t-1} tile
+  tile_mainloop<BF16G>(p1, L1, false, r, 1, R1, false, n, 1, m, n, r, i0, j0, Xs, Ys);   // P_t tile
+
+  float* W = static_cast<float*>(b.p[BASE_PARAMS]) + A.off;
+  const void* G = static_cast<const char*>(b.p[BASE_GRADS]) + (size_t)A.off * (BF16G ? 2 : 4);
+  float* V = state + A.v_off;
+  const float lr_s = sc.lr * A.lr_scale;
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+#pragma unroll
+  for (int rr = 0; rr < 4; ++rr) {
+    const int i = i0 + ty * 4 + rr;
+    if (i >= m) continue;
+    float v_row = 0.f;
+    if (A.v_mode == ADAPM_V_BLOCKMEAN) v_row = V[i / A.v_group_rows];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int j = j0 + tx * 4 + c;
+      if (j >= n) continue;
+      const int64_t o = (int64_t)i * n + j;
+      const float g = load_operand<BF16G>(G, true, o);
+      const float mc = sc.cg * g + sc.c0 * p0[rr][c] - sc.c1 * p1[rr][c];
+      float v = v_row;
+      if (A.v_mode == ADAPM_V_ELEMENT) {
+        v = sc.beta2 * V[o] + (1.f - sc.beta2) * (g * g);
+        V[o] = v;
+      }
+      W[o] = adapm_param_update(W[o], mc, v, sc, lr_s, A.wd);
+    }
+  }
+}
+
+// ---- L_0: Gaussian draws, then modified Gram-Schmidt, one CTA per block ------------------------
+
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__device__ __forceinline__ float gaussian_from_counter(uint64_t seed, uint64_t block, uint64_t idx) {
+  const uint64_t h = mix64(mix64(seed ^ (block * 0xD1342543DE82EF95ull)) + idx);
+  const float u1 = ((uint32_t)(h >> 40) + 1.0f) * (1.0f / 16777217.0f);   // (0, 1)
+  const float u2 = (uint32_t)(h & 0xFFFFFFu) * (1.0f / 16777216.0f);       // [0, 1)
+  return sqrtf(-2.f * logf(u1)) * cosf(6.283185307179586f * u2);
+}
+
+__device__ __forceinline__ float block_sum_1024(float x, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+  __syncthreads();
+  float s = 0.f;
+  const int nw = blockDim.x >> 5;
+  for (int i = 0; i < nw; ++i) s += red[i];
+  return s;
+}
+
+__global__ void __launch_bounds__(1024) init_L0_kernel(const InitJob* __restrict__ tab, float* __restrict__ state,
+                                                       uint64_t seed) {
+  __shared__ float red[32];
+  const InitJob J = tab[blockIdx.x];
+  float* __restrict__ L = state + J.l_off;
+  const int rows = J.rows, rank = J.rank;
+  const uint64_t block = (uint64_t)J.block_index;
+  const int64_t total = (int64_t)rows * rank;
+  for (int64_t e = threadIdx.x; e < total; e += blockDim.x) L[e] = gaussian_from_counter(seed, block, (uint64_t)e);
+  __syncthreads();
+  for (int j = 0; j < rank; ++j) {
+    for (int i = 0; i < j; ++i) {
+      float d = 0.f;
+      for (int row = threadIdx.x; row < rows; row += blockDim.x) d += L[(int64_t)row * rank + i] * L[(int64_t)row * rank + j];
+      d = block_sum_1024(d, red);
+      for (int row = threadIdx.x; row < rows; row += blockDim.x) L[(int64_t)row * rank + j] -= d * L[(int64_t)row * rank + i];
+    }
+    float nn = 0.f;
+    for (int row = threadIdx.x; row < rows; row += blockDim.x) {
+      const float x = L[(int64_t)row * rank + j];
+      nn += x * x;
+    }
+    nn = block_sum_1024(nn, red);
+    const float inv = rsqrtf(nn);
+    for (int row = threadIdx.x; row < rows; row += blockDim.x) L[(int64_t)row * rank + j] *= inv;
+    __syncthreads();
+  }
+}
+
+}  // namespace
+
+#define ADAPM_LAUNCH_CHECK()                         \
+  do {                                               \
+    cudaError_t e__ = cudaGetLastError();            \
+    if (e__ != cudaSuccess) {                        \
+      set_cuda_error(e__, __func__);                 \
+      return ADAPM_ECUDA;                            \
+    }                                                \
+  } while (0)
+
+int launch_gemm(const GemmProb* d_tab, int64_t n_prob, int64_t n_tiles, const Bases& b, int grad_dtype,
+                cudaStream_t s) {
+  if (n_tiles <= 0) return ADAPM_OK;
+  if (grad_dtype == ADAPM_GRAD_BF16)
+    gemm_kernel<true><<<(unsigned)n_tiles, 256, 0, s>>>(d_tab, (int)n_prob, b);
+  else
+    gemm_kernel<false><<<(unsigned)n_tiles, 256, 0, s>>>(d_tab, (int)n_prob, b);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_apply_simt(const ApplyBlk* d_tab, int64_t n_blk, int64_t n_tiles, const Bases& b, const StepScalars& sc,
+                      int grad_dtype, cudaStream_t s) {
+  if (n_tiles <= 0) return ADAPM_OK;
+  if (grad_dtype == ADAPM_GRAD_BF16)
+    apply_simt_kernel<true><<<(unsigned)n_tiles, 256, 0, s>>>(d_tab, (int)n_blk, b, sc);
+  else
+    apply_simt_kernel<false><<<(unsigned)n_tiles, 256, 0, s>>>(d_tab, (int)n_blk, b, sc);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_init_L0(const InitJob* d_tab, int64_t n_jobs, float* state, uint64_t seed, cudaStream_t s) {
+  if (n_jobs <= 0) return ADAPM_OK;
+  init_L0_kernel<<<(unsigned)n_jobs, 1024, 0, s>>>(d_tab, state, seed);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+}  // namespace adapm

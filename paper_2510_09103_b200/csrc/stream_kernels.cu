@@ -1,0 +1,368 @@
+// Fused streaming update for blocks without momentum and with full momentum, and the block-mean
+// reduction of g^2 for second-moment groups that do not fit one team of threads.
+//
+// Per element the kernel performs, in one pass over HBM (Algorithm 1 lines 7 and 9, Eq. 4):
+//   v  <- beta2 v + (1-beta2) g^2            (per element, or once per group with the group mean of g^2)
+//   m  <- beta1 m + (1-beta1) g              (full-momentum blocks only; m^c = m, else m^c = g)
+//   W  <- W - lr s_b ( clamp( m^c / (sqrt(v)+eps) ) + lambda_b W )
+// A work unit (one v group, or a 2048-element chunk) is owned by a team of 32 or 256 threads that
+// keeps the unit's gradient in registers, so g is read from memory exactly once even when the
+// group mean has to be known before any element can be updated.
+#include "adapm_internal.h"
+#include "device_math.cuh"
+
+namespace adapm {
+
+namespace {
+
+template <int TEAM>
+__device__ __forceinline__ float team_sum(float x, float* smem8) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  if (TEAM == 32) return x;
+  const int w = threadIdx.x >> 5;
+  __syncthreads();                       // smem8 may still be read from a previous use
+  if ((threadIdx.x & 31) == 0) smem8[w] = x;
+  __syncthreads();
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s += smem8[i];   // same order in every thread
+  return s;
+}
+
+template <typename GT, int TEAM>
+__device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float* __restrict__ params,
+                                         const typename GT::elem* __restrict__ grads, float* __restrict__ state,
+                                         const StepScalars& sc, float* smem8) {
+  const int lane = (TEAM == 32) ? (threadIdx.x & 31) : threadIdx.x;
+
+  int64_t ustart, group;
+  int ulen;
+  if (B.v_mode == SV_GROUP_READY) {
+    group = unit / B.units_per_group;
+    const int64_t u = unit - group * B.units_per_group;
+    const int64_t in_group = u * B.unit_elems;
+    ustart = group * B.group_elems + in_group;
+    const int64_t rem = B.group_elems - in_group;
+    ulen = rem < B.unit_elems ? (int)rem : B.unit_elems;
+  } else {
+    group = unit;
+    ustart = unit * (int64_t)B.unit_elems;
+    const int64_t rem = B.numel - ustart;
+    ulen = rem < B.unit_elems ? (int)rem : B.unit_elems;
+  }
+  const typename GT::elem* g = grads + B.off + ustart;
+  float* W = params + B.off + ustart;
+  float* M = (B.m_off >= 0) ? state + B.m_off + ustart : nullptr;
+  const int nchunks = (ulen + kChunkElems - 1) / kChunkElems;
+  const bool vec = B.vec_ok != 0;
+
+  // ---- phase 1: gradient into registers, sum of squares --------------------------------------
+  typename GT::raw8 graw[kTeamChunks];
+  float ss = 0.f;
+#pragma unroll
+  for (int c = 0; c < kTeamChunks; ++c) {
+    const int idx = lane + c * TEAM;
+    if (idx < nchunks) {
+      const int e0 = idx * kChunkElems;
+      if (vec && e0 + kChunkElems <= ulen) {
+        graw[c] = GT::load8(g + e0);
+      } else {
+        graw[c] = GT::load8_guarded(g + e0, ulen - e0);
+      }
+      float f[8];
+      GT::unpack(graw[c], f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+    }
+  }
+
+  float v_group = 0.f;
+  if (B.v_mode == SV_GROUP_INLINE) {
+    // one thread reads the old scalar and writes the new one; everyone else gets it by broadcast
+    float v_old = 0.f;
+    if (lane == 0) v_old = state[B.v_off + group];
+    const float tot = team_sum<TEAM>(ss, smem8);
+    if (TEAM == 32) {
+      v_old = __shfl_sync(0xffffffffu, v_old, 0);
+    } else {
+      if (threadIdx.x == 0) smem8[8] = v_old;
+      __syncthreads();
+      v_old = smem8[8];
+    }
+    v_group = sc.beta2 * v_old + (1.f - sc.beta2) * (tot / (float)ulen);
+    if (lane == 0) state[B.v_off + group] = v_group;
+  } else if (B.v_mode == SV_GROUP_READY) {
+    v_group = state[B.v_off + group];
+  }
+  float* V = (B.v_mode == SV_ELEMENT) ? state + B.v_off + ustart : nullptr;
+
+  // ---- phase 2: momentum, second moment, parameter write ------------------------------------
+  const float lr_s = sc.lr * B.lr_scale;
+  const float a1 = 1.f - sc.beta1, a2 = 1.f - sc.beta2;
+#pragma unroll
+  for (int c = 0; c < kTeamChunks; ++c) {
+    const int idx = lane + c * TEAM;
+    if (idx < nchunks) {
+      const int e0 = idx * kChunkElems;
+      const bool full = vec && e0 + kChunkElems <= ulen;
+      const int nval = full ? 8 : (ulen - e0 < 8 ? ulen - e0 : 8);
+      float gf[8], w[8], m[8], v[8];
+      GT::unpack(graw[c], gf);
+      if (full) {
+        load8f(W + e0, w);
+        if (M) load8f(M + e0, m);
+        if (V) load8f(V + e0, v);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const bool ok = i < nval;
+          w[i] = ok ? W[e0 + i] : 0.f;
+          m[i] = (ok && M) ? M[e0 + i] : 0.f;
+          v[i] = (ok && V) ? V[e0 + i] : 0.f;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float mc = gf[i];
+        if (M) {
+          m[i] = sc.beta1 * m[i] + a1 * gf[i];
+          mc = m[i];
+        }
+        float vv = v_group;
+        if (V) {
+          v[i] = sc.beta2 * v[i] + a2 * (gf[i] * gf[i]);
+          vv = v[i];
+        }
+        w[i] = adapm_param_update(w[i], mc, vv, sc, lr_s, B.wd);
+      }
+      if (full) {
+        store8f(W + e0, w);
+        if (M) store8f(M + e0, m);
+        if (V) store8f(V + e0, v);
+      } else {
+        for (int i = 0; i < nval; ++i) {
+          W[e0 + i] = w[i];
+          if (M) M[e0 + i] = m[i];
+          if (V) V[e0 + i] = v[i];
+        }
+      }
+    }
+  }
+}
+
+template <typename GT>
+__global__ void __launch_bounds__(256) stream_update_kernel(const StreamBlk* __restrict__ tab, int n_blk,
+                                                            float* __restrict__ params,
+                                                            const typename GT::elem* __restrict__ grads,
+                                                            float* __restrict__ state, StepScalars sc) {
+  __shared__ StreamBlk sB;
+  __shared__ float smem8[12];
+  if (threadIdx.x == 0) {
+    int lo = 0, hi = n_blk - 1;            // last block with first_cta <= blockIdx.x
+    const int64_t me = blockIdx.x;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (tab[mid].first_cta <= me) lo = mid; else hi = mid - 1;
+    }
+    sB = tab[lo];
+  }
+  __syncthreads();
+  const int64_t cta_local = (int64_t)blockIdx.x - sB.first_cta;
+  if (sB.team == 32) {
+    const int64_t unit = cta_local * 8 + (threadIdx.x >> 5);
+    if (unit < sB.n_units) run_unit<GT, 32>(sB, unit, params, grads, state, sc, smem8);
+  } else {
+    run_unit<GT, 256>(sB, cta_local, params, grads, state, sc, smem8);
+  }
+}
+
+// ---- group sums of squares ---------------------------------------------------------------------
+
+template <typename GT>
+__device__ __forceinline__ float warp_chunk_sumsq(const typename GT::elem* __restrict__ g, int len, bool vec) {
+  const int lane = threadIdx.x & 31;
+  const int nchunks = (len + kChunkElems - 1) / kChunkElems;
+  float ss = 0.f;
+#pragma unroll
+  for (int c = 0; c < kTeamChunks; ++c) {
+    const int idx = lane + c * 32;
+    if (idx < nchunks) {
+      const int e0 = idx * kChunkElems;
+      typename GT::raw8 r = (vec && e0 + kChunkElems <= len) ? GT::load8(g + e0) : GT::load8_guarded(g + e0, len - e0);
+      float f[8];
+      GT::unpack(r, f);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  return ss;
+}
+
+template <typename GT>
+__global__ void __launch_bounds__(256) reduce_partial_kernel(const ReduceJob* __restrict__ tab, int n_jobs,
+                                                             int64_t n_units,
+                                                             const typename GT::elem* __restrict__ grads,
+                                                             float* __restrict__ work) {
+  const int64_t unit = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (unit >= n_units) return;
+  int lo = 0, hi = n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (tab[mid].first_unit <= unit) lo = mid; else hi = mid - 1;
+  }
+  const ReduceJob J = tab[lo];
+  const int64_t u = unit - J.first_unit;
+  const int64_t group = u / J.chunks_per_group;
+  const int64_t chunk = u - group * J.chunks_per_group;
+  const int64_t in_group = chunk * kWarpUnitMax;
+  const int64_t rem = J.group_elems - in_group;
+  const int len = rem < kWarpUnitMax ? (int)rem : kWarpUnitMax;
+  const bool vec = (J.group_elems % kChunkElems) == 0 || J.n_groups == 1;
+  const float ss = warp_chunk_sumsq<GT>(grads + J.g_off + group * J.group_elems + in_group, len, vec);
+  if ((threadIdx.x & 31) == 0) work[J.part_off + u] = ss;
+}
+
+__device__ __forceinline__ float warp_sum_partials(const float* __restrict__ p, int n) {
+  const int lane = threadIdx.x & 31;
+  float s = 0.f;
+  for (int i = lane; i < n; i += 32) s += p[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  return s;
+}
+
+__global__ void __launch_bounds__(256) reduce_final_kernel(const ReduceJob* __restrict__ tab, int n_jobs,
+                                                           int64_t n_groups, float* __restrict__ state,
+                                                           const float* __restrict__ work, float beta2) {
+  const int64_t gidx = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (gidx >= n_groups) return;
+  int lo = 0, hi = n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (tab[mid].first_group <= gidx) lo = mid; else hi = mid - 1;
+  }
+  const ReduceJob J = tab[lo];
+  const int64_t group = gidx - J.first_group;
+  const float tot = warp_sum_partials(work + J.part_off + group * J.chunks_per_group, J.chunks_per_group);
+  if ((threadIdx.x & 31) == 0) {
+    float* v = state + J.v_off + group;
+    *v = beta2 * (*v) + (1.f - beta2) * (tot / (float)J.group_elems);
+  }
+}
+
+// stand-alone block mean of g^2 (same two stages, caller's scratch)
+template <typename GT>
+__global__ void __launch_bounds__(256) meansq_partial_kernel(const typename GT::elem* __restrict__ g,
+                                                             int64_t n_groups, int64_t group_elems,
+                                                             int chunks_per_group, float* __restrict__ partial) {
+  const int64_t unit = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (unit >= n_groups * chunks_per_group) return;
+  const int64_t group = unit / chunks_per_group;
+  const int64_t chunk = unit - group * chunks_per_group;
+  const int64_t in_group = chunk * kWarpUnitMax;
+  const int64_t rem = group_elems - in_group;
+  const int len = rem < kWarpUnitMax ? (int)rem : kWarpUnitMax;
+  const bool vec = (group_elems % kChunkElems) == 0 || n_groups == 1;
+  const float ss = warp_chunk_sumsq<GT>(g + group * group_elems + in_group, len, vec);
+  if ((threadIdx.x & 31) == 0) partial[unit] = ss;
+}
+
+__global__ void __launch_bounds__(256) meansq_final_kernel(const float* __restrict__ partial, int64_t n_groups,
+                                                           int64_t group_elems, int chunks_per_group,
+                                                           float* __restrict__ out) {
+  const int64_t group = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (group >= n_groups) return;
+  const float tot = warp_sum_partials(partial + group * chunks_per_group, chunks_per_group);
+  if ((threadIdx.x & 31) == 0) out[group] = tot / (float)group_elems;
+}
+
+__global__ void copy_f32_kernel(float4* __restrict__ dst, const float4* __restrict__ src, int64_t n4) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
+}  // namespace
+
+#define ADAPM_LAUNCH_CHECK()                         \
+  do {                                               \
+    cudaError_t e__ = cudaGetLastError();            \
+    if (e__ != cudaSuccess) {                        \
+      set_cuda_error(e__, __func__);                 \
+      return ADAPM_ECUDA;                            \
+    }                                                \
+  } while (0)
+
+int launch_stream(const StreamBlk* d_tab, int64_t n_blk, int64_t grid, const Bases& b, const StepScalars& sc,
+                  int grad_dtype, cudaStream_t s) {
+  if (grid <= 0) return ADAPM_OK;
+  if (grad_dtype == ADAPM_GRAD_BF16)
+    stream_update_kernel<GradBF16><<<(unsigned)grid, 256, 0, s>>>(d_tab, (int)n_blk, (float*)b.p[BASE_PARAMS],
+                                                                 (const uint16_t*)b.p[BASE_GRADS],
+                                                                 (float*)b.p[BASE_STATE], sc);
+  else
+    stream_update_kernel<GradF32><<<(unsigned)grid, 256, 0, s>>>(d_tab, (int)n_blk, (float*)b.p[BASE_PARAMS],
+                                                                (const float*)b.p[BASE_GRADS],
+                                                                (float*)b.p[BASE_STATE], sc);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_reduce_partial(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_units, const void* grads, float* work,
+                          int grad_dtype, cudaStream_t s) {
+  if (n_units <= 0) return ADAPM_OK;
+  const unsigned grid = (unsigned)((n_units + 7) / 8);
+  if (grad_dtype == ADAPM_GRAD_BF16)
+    reduce_partial_kernel<GradBF16><<<grid, 256, 0, s>>>(d_tab, (int)n_jobs, n_units, (const uint16_t*)grads, work);
+  else
+    reduce_partial_kernel<GradF32><<<grid, 256, 0, s>>>(d_tab, (int)n_jobs, n_units, (const float*)grads, work);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_reduce_final(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_groups, float* state, const float* work,
+                        float beta2, cudaStream_t s) {
+  if (n_groups <= 0) return ADAPM_OK;
+  reduce_final_kernel<<<(unsigned)((n_groups + 7) / 8), 256, 0, s>>>(d_tab, (int)n_jobs, n_groups, state, work, beta2);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_meansq_partial(const void* g, int grad_dtype, int64_t n_groups, int64_t group_elems, int chunks_per_group,
+                          float* partial, cudaStream_t s) {
+  const int64_t units = n_groups * chunks_per_group;
+  if (units <= 0) return ADAPM_OK;
+  const unsigned grid = (unsigned)((units + 7) / 8);
+  if (grad_dtype == ADAPM_GRAD_BF16)
+    meansq_partial_kernel<GradBF16><<<grid, 256, 0, s>>>((const uint16_t*)g, n_groups, group_elems, chunks_per_group,
+                                                         partial);
+  else
+    meansq_partial_kernel<GradF32><<<grid, 256, 0, s>>>((const float*)g, n_groups, group_elems, chunks_per_group,
+                                                        partial);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_meansq_final(const float* partial, int64_t n_groups, int64_t group_elems, int chunks_per_group, float* out,
+                        cudaStream_t s) {
+  if (n_groups <= 0) return ADAPM_OK;
+  meansq_final_kernel<<<(unsigned)((n_groups + 7) / 8), 256, 0, s>>>(partial, n_groups, group_elems, chunks_per_group,
+                                                                    out);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_copy_f32(float* dst, const float* src, int64_t n, cudaStream_t s) {
+  if (n <= 0) return ADAPM_OK;
+  // n is a multiple of 64 floats by construction of the state layout
+  const int64_t n4 = n / 4;
+  int64_t grid = (n4 + 255) / 256;
+  if (grid > 148 * 16) grid = 148 * 16;
+  copy_f32_kernel<<<(unsigned)grid, 256, 0, s>>>((float4*)dst, (const float4*)src, n4);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+}  // namespace adapm
