@@ -32,8 +32,9 @@ def rel_err(gpu: np.ndarray, ref: np.ndarray) -> float:
 
 
 def oracle_blocks_from(blocks: Sequence) -> List[O.Block]:
+    # lr_scale / weight_decay are fp32 fields of the descriptor: the oracle sees exactly those values
     return [O.Block(rows=b.rows, cols=b.cols, mom_mode=b.mom_mode, rank=b.rank, v_mode=b.v_mode,
-                    v_group_rows=b.v_group_rows, lr_scale=b.lr_scale, weight_decay=b.weight_decay,
+                    v_group_rows=b.v_group_rows, lr_scale=float(b.lr_scale), weight_decay=float(b.weight_decay),
                     offset=b.offset) for b in blocks]
 
 
@@ -113,8 +114,10 @@ class ParityRun:
         self.ctx.adapm_state_init(self.state)
 
         # oracle side: its own L_0, injected into the GPU state so that both start from the same factors
-        oh = O.HParams(lr=hpk["lr"], beta1=hpk["beta1"], beta2=hpk["beta2"], eps=hpk["eps"], clip=hpk["clip"],
-                       inner_iters=hpk["inner_iters"], inner_lr_scale=hpk["inner_lr_scale"],
+        # the C ABI takes its hyperparameters as fp32: the oracle gets the same (rounded) values
+        f32 = lambda x: float(np.float32(x))
+        oh = O.HParams(lr=f32(hpk["lr"]), beta1=f32(hpk["beta1"]), beta2=f32(hpk["beta2"]), eps=f32(hpk["eps"]),
+                       clip=f32(hpk["clip"]), inner_iters=hpk["inner_iters"], inner_lr_scale=f32(hpk["inner_lr_scale"]),
                        adam_debias=bool(hpk.get("adam_debias", 0)), correction=bool(hpk.get("correction", 1)))
         self.ohp = oh
         self.ostate: Dict[int, O.BlockState] = {}
