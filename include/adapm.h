@@ -175,6 +175,30 @@ size_t adapm_group_meansq_scratch_bytes(int64_t n_groups, int64_t group_elems);
 int adapm_group_meansq(const void* g, int32_t grad_dtype, int64_t n_groups, int64_t group_elems,
                        float* out, void* scratch, size_t scratch_bytes, adapm_stream stream);
 
+/*
+ * adapm_group_meansq without any device allocation (the paper has no counterpart; this is a
+ * packaging variant of the call above for callers that must not, or cannot, call cudaMalloc:
+ * code running inside a host application whose memory manager owns the whole GPU, plug-ins
+ * that are forbidden to allocate in their callback, and loops that cannot afford the implicit
+ * device synchronisation an allocation or free may cause).
+ *
+ * Same arguments and result as adapm_group_meansq, minus the scratch: the partial sums go to a
+ * fixed array of ADAPM_STATIC_SCRATCH_FLOATS floats (1 MiB) that is part of the library image;
+ * every GPU that loads the library keeps that array until the process exits.
+ *   - Limit: n_groups * ceil(group_elems / 2048) <= ADAPM_STATIC_SCRATCH_FLOATS, else ADAPM_ERANGE
+ *     (adapm_last_cuda_error() then says so); larger inputs need adapm_group_meansq.
+ *   - The call itself allocates and frees nothing.  Its first call on each device looks up the
+ *     array's device address (one cudaGetSymbolAddress, with that device current): make that first
+ *     call before starting any stream capture.  `stream` must belong to the current device.
+ *   - All calls on a device share the one array.  Calls whose kernels may overlap on the GPU
+ *     (different streams without an ordering between them) race on it: order them on one stream
+ *     or with events.  Nothing has to be cleared between calls: each call overwrites the part of
+ *     the array it then reads.
+ */
+#define ADAPM_STATIC_SCRATCH_FLOATS (1 << 18)
+int adapm_group_meansq_static(const void* g, int32_t grad_dtype, int64_t n_groups, int64_t group_elems,
+                              float* out, adapm_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

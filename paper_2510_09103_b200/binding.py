@@ -24,7 +24,7 @@ EXPORTS = (
     "adapm_workspace_bytes", "adapm_set_workspace", "adapm_state_init", "adapm_set_lr", "adapm_step",
     "adapm_step_bytes", "adapm_step_flops", "adapm_launch_count", "adapm_get_status",
     "adapm_group_meansq_scratch_bytes", "adapm_group_meansq", "adapm_set_profiling", "adapm_get_launch_times",
-    "adapm_launch_kind_name",
+    "adapm_launch_kind_name", "adapm_group_meansq_static",
 )
 
 
@@ -104,6 +104,7 @@ def load(build_if_missing: bool = True) -> C.CDLL:
         "adapm_get_status": (C.c_int, [vp, vp, C.POINTER(i32)]),
         "adapm_group_meansq_scratch_bytes": (sz, [i64, i64]),
         "adapm_group_meansq": (C.c_int, [vp, i32, i64, i64, vp, vp, sz, vp]),
+        "adapm_group_meansq_static": (C.c_int, [vp, i32, i64, i64, vp, vp]),
         "adapm_set_profiling": (C.c_int, [vp, i32]),
         "adapm_get_launch_times": (C.c_int, [vp, C.POINTER(C.c_float), C.POINTER(i32), i64, C.POINTER(i64)]),
         "adapm_launch_kind_name": (C.c_char_p, [i32]),
@@ -266,3 +267,14 @@ def adapm_group_meansq(g, grad_dtype: int, n_groups: int, group_elems: int, out,
     nbytes = scratch.numel() * scratch.element_size()
     _check(load().adapm_group_meansq(_ptr(g), grad_dtype, n_groups, group_elems, _ptr(out), _ptr(scratch), nbytes,
                                      _stream(stream)), "adapm_group_meansq")
+
+
+STATIC_SCRATCH_FLOATS = 1 << 18
+
+
+def adapm_group_meansq_static(g, grad_dtype: int, n_groups: int, group_elems: int, out, stream=None) -> None:
+    """Block mean of g^2 with the library's built-in scratch: for callers that must not allocate device
+    memory.  Limit: n_groups * ceil(group_elems / 2048) <= STATIC_SCRATCH_FLOATS.  Calls that may overlap
+    on the GPU share the scratch and race; keep them on one stream."""
+    _check(load().adapm_group_meansq_static(_ptr(g), grad_dtype, n_groups, group_elems, _ptr(out), _stream(stream)),
+           "adapm_group_meansq_static")

@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libadapm.so")
-SOURCES = ["planner.cpp", "ctx.cu", "stream_kernels.cu", "lowrank_simt.cu", "lowrank_tc.cu"]
+SOURCES = ["planner.cpp", "ctx.cu", "stream_kernels.cu", "lowrank_simt.cu", "lowrank_tc.cu", "static_scratch.cu"]
 
 
 def _nvcc() -> str:

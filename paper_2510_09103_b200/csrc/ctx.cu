@@ -16,6 +16,8 @@ void set_cuda_error(cudaError_t e, const char* where) {
   g_cuda_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " at " + where;
 }
 
+void set_error_text(const char* text) { g_cuda_error = text ? text : ""; }
+
 namespace {
 
 template <typename T>
