@@ -129,7 +129,7 @@ struct StepScalars {
 // one launch of the static per-step program
 enum LaunchKind : int32_t {
   LK_REDUCE_PARTIAL, LK_REDUCE_FINAL, LK_STREAM, LK_GEMM, LK_APPLY_SIMT, LK_COMMIT,
-  LK_TC_CONVERT, LK_TC_PANEL, LK_TC_UPDATE, LK_TC_APPLY
+  LK_TC_CONVERT, LK_TC_GRAM, LK_TC_PANEL, LK_TC_APPLY
 };
 struct Launch {
   LaunchKind kind;
@@ -159,6 +159,8 @@ int launch_meansq_final(const float* partial, int64_t n_groups, int64_t group_el
                         cudaStream_t s);
 int launch_init_L0(const InitJob* d_tab, int64_t n_jobs, float* state, uint64_t seed, cudaStream_t s);
 
+struct TcProgram;   // host side of the tensor-core low-rank path (lowrank_tc.cu)
+
 }  // namespace adapm
 
 // The opaque context.
@@ -170,7 +172,7 @@ struct adapm_ctx {
   // state layout (floats)
   std::vector<int64_t> m_off, l_off, r_off, v_off, v_cnt;
   int64_t state_floats = 0;
-  int64_t lr_section_floats = 0;       // the L,R section sits at the start of the state buffer
+  int64_t lr_section_floats = 0;       // L,R of the CUDA-core blocks: the start of the state buffer
   size_t bytes_m = 0, bytes_L = 0, bytes_R = 0, bytes_v = 0;
 
   // workspace layout (floats)
@@ -186,7 +188,8 @@ struct adapm_ctx {
   int32_t* d_status = nullptr;
   int64_t init_table_off = 0, n_init_jobs = 0;
   int final_lr_buf = -1;               // which workspace copy holds L_t,R_t after the refit (-1: unchanged)
-  int use_tensor_path = 0;
+  adapm::TcProgram* tc = nullptr;      // program of the blocks that run on the tensor cores
+  int64_t n_tensor_blocks = 0;
 
   // optional per-launch timing (adapm_set_profiling)
   int profiling = 0, prof_valid = 0;

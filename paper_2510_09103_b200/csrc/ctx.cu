@@ -64,10 +64,12 @@ int validate(const adapm_block* blocks, int64_t n, const adapm_hparams& hp) {
 
 }  // namespace
 
-// builds the tensor-core program for the low-rank blocks; defined in lowrank_tc.cu
-int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& lowrank_ids, int64_t& work_cursor);
+// the tensor-core program of the low-rank blocks; defined in lowrank_tc.cu
+bool tensor_path_block_ok(const adapm_hparams& hp, const adapm_block& b);
+int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const std::vector<double>& etas,
+                         int64_t& work_cursor);
+int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s);
 int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepScalars& sc, cudaStream_t s);
-bool tensor_path_supports(const adapm_ctx* c, const std::vector<int64_t>& lowrank_ids);
 void destroy_tensor_program(adapm_ctx* c);
 
 }  // namespace adapm
@@ -89,20 +91,31 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   const int n = (int)n_blocks;
   const size_t gsz = hp->grad_dtype == ADAPM_GRAD_BF16 ? 2 : 4;
 
-  // ---- state layout: [L,R of every low-rank block][m^f of every full block][v of every block] ----
-  c->m_off.assign(n, -1); c->l_off.assign(n, -1); c->r_off.assign(n, -1); c->v_off.assign(n, -1); c->v_cnt.assign(n, 0);
-  int64_t cur = 0;
-  std::vector<int64_t> lowrank_ids;
+  // ---- which kernels run each low-rank block ----------------------------------------------------------
+  std::vector<int64_t> lowrank_ids, tc_ids;     // lowrank_ids: the blocks of the CUDA-core path
   for (int i = 0; i < n; ++i) {
     const adapm_block& b = c->blocks[i];
     if (b.mom_mode != ADAPM_MOM_LOWRANK) continue;
-    lowrank_ids.push_back(i);
+    if (tensor_path_block_ok(*hp, b)) tc_ids.push_back(i);
+    else if (hp->lowrank_path == ADAPM_PATH_TENSOR) { delete c; return ADAPM_EUNSUPPORTED; }
+    else lowrank_ids.push_back(i);
+  }
+  c->n_tensor_blocks = (int64_t)tc_ids.size();
+
+  // ---- state layout: [L,R of the CUDA-core low-rank blocks][L,R of the tensor-core ones]
+  //                    [m^f of every full block][v of every block] --------------------------------------
+  c->m_off.assign(n, -1); c->l_off.assign(n, -1); c->r_off.assign(n, -1); c->v_off.assign(n, -1); c->v_cnt.assign(n, 0);
+  int64_t cur = 0;
+  auto place_factors = [&](int64_t i) {
+    const adapm_block& b = c->blocks[i];
     c->l_off[i] = cur; cur += round_up((int64_t)b.rows * b.rank, kStateAlign);
     c->r_off[i] = cur; cur += round_up((int64_t)b.rank * b.cols, kStateAlign);
     c->bytes_L += (size_t)b.rows * b.rank * 4;
     c->bytes_R += (size_t)b.rank * b.cols * 4;
-  }
+  };
+  for (int64_t i : lowrank_ids) place_factors(i);
   c->lr_section_floats = cur;
+  for (int64_t i : tc_ids) place_factors(i);
   for (int i = 0; i < n; ++i) {
     const adapm_block& b = c->blocks[i];
     if (b.mom_mode != ADAPM_MOM_FULL) continue;
@@ -186,17 +199,9 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     sblk.push_back(s);
   }
 
-  // ---- which path runs the low-rank blocks ---------------------------------------------------------
-  c->use_tensor_path = 0;
-  if (!lowrank_ids.empty() && hp->lowrank_path != ADAPM_PATH_SIMT) {
-    const bool ok = tensor_path_supports(c, lowrank_ids);
-    if (ok) c->use_tensor_path = 1;
-    else if (hp->lowrank_path == ADAPM_PATH_TENSOR) { delete c; return ADAPM_EUNSUPPORTED; }
-  }
-
-  // SIMT path: group sums of g^2 of low-rank blocks come from the reduction kernels
-  if (!c->use_tensor_path) {
-    for (int64_t i : lowrank_ids) {
+  // group sums of g^2 of the low-rank blocks come from the reduction kernels
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int64_t i : (pass == 0 ? lowrank_ids : tc_ids)) {
       const adapm_block& b = c->blocks[i];
       if (b.v_mode != ADAPM_V_BLOCKMEAN) continue;
       const int64_t numel = (int64_t)b.rows * b.cols;
@@ -217,16 +222,19 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   }
 
   // ---- low-rank program --------------------------------------------------------------------------
-  if (!lowrank_ids.empty()) {
+  if (!lowrank_ids.empty() || !tc_ids.empty()) {
     std::vector<InitJob> ijobs;
-    for (int64_t i : lowrank_ids) ijobs.push_back({c->l_off[i], i, c->blocks[i].rows, c->blocks[i].rank});
+    for (int pass = 0; pass < 2; ++pass)
+      for (int64_t i : (pass == 0 ? lowrank_ids : tc_ids))
+        ijobs.push_back({c->l_off[i], i, c->blocks[i].rows, c->blocks[i].rank});
     c->init_table_off = append_table(c->h_tables, ijobs);
     c->n_init_jobs = (int64_t)ijobs.size();
   }
-  if (!lowrank_ids.empty() && c->use_tensor_path) {
-    rc = build_tensor_program(c, lowrank_ids, work_cursor);
-    if (rc != ADAPM_OK) { delete c; return rc; }
-  } else if (!lowrank_ids.empty()) {
+  if (!tc_ids.empty()) {
+    rc = build_tensor_program(c, tc_ids, etas, work_cursor);
+    if (rc != ADAPM_OK) { adapm_destroy(c); return rc; }
+  }
+  if (!lowrank_ids.empty()) {
     // workspace: two copies of the [L,R] section (ping-pong iterates), A/B with the same layout, Gram matrices
     c->ws_lr[0] = work_cursor; work_cursor += c->lr_section_floats;
     c->ws_lr[1] = work_cursor; work_cursor += c->lr_section_floats;
@@ -446,6 +454,10 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
   b.p[BASE_WORK] = c->workspace;
   float* work = (float*)c->workspace;
 
+  if (c->tc) {
+    const int prc = tensor_prepare_step(c, b, s);
+    if (prc != ADAPM_OK) return prc;
+  }
   const bool prof = c->profiling && c->prof_events.size() == c->program.size() + 1;
   if (prof) ADAPM_CUDA(cudaEventRecord(c->prof_events[0], s));
   size_t li = 0;
@@ -511,7 +523,7 @@ extern "C" const char* adapm_launch_kind_name(int32_t kind) {
     case LK_COMMIT: return "commit_copy";
     case LK_TC_CONVERT: return "tc_convert";
     case LK_TC_PANEL: return "tc_panel";
-    case LK_TC_UPDATE: return "tc_update";
+    case LK_TC_GRAM: return "tc_gram";
     case LK_TC_APPLY: return "tc_apply";
     default: return "unknown";
   }

@@ -1,13 +1,411 @@
-// Tensor-core (tcgen05) kernels of the low-rank path.
+// Tensor-core (tcgen05) low-rank path: the per-step program of Algorithm 2's refit and of the
+// corrected update for every low-rank block whose layout the TMA engine can address
+// (bf16 gradients, cols a multiple of 8, rank <= 128).
+//
+// Per step:
+//   convert   (L_{t-1}, R_{t-1}) fp32 -> split-bf16 arrays  Lc[0] = [L hi | L lo]  (rows x 2rp)
+//                                                           RTc[0] = [R^T hi | R^T lo] (cols x 2rp)
+//   K_eff times:  gram    four r x r products of the current iterate (tensor cores) -> Gs[0..3]
+//                 panel   row panels update L, column panels update R (tensor cores); fp32 factors
+//                         are updated in place in the state, their split copies go to the other of
+//                         the two iterate sets Lc[1|2], RTc[1|2]
+//   apply     m^c and the parameter write from (Lc[0], RTc[0]) and the final iterate set
+// rp = rank rounded up to 16; padded columns are kept at zero by every writer.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+
 #include "adapm_internal.h"
+#include "tc_apply.cuh"
+#include "tc_engine.cuh"
+#include "tc_host.h"
 
 namespace adapm {
 
-bool tensor_path_supports(const adapm_ctx*, const std::vector<int64_t>&) { return false; }
-int build_tensor_program(adapm_ctx*, const std::vector<int64_t>&, int64_t&) { return ADAPM_EUNSUPPORTED; }
-int run_tensor_launch(adapm_ctx*, const Launch&, const Bases&, const StepScalars&, cudaStream_t) {
-  return ADAPM_EUNSUPPORTED;
+void set_error_text(const char* text);   // ctx.cu
+
+namespace {
+
+constexpr int kMapsPerBlock = 11;   // g, Lc[3], RTc[3], Gs[4]
+enum { MAP_G = 0, MAP_LC = 1, MAP_RTC = 4, MAP_GS = 7 };
+
+struct ConvertJob {
+  int64_t f32_off;          // float offset of the factor in state
+  int64_t own_stride, k_stride;
+  int64_t dst_off;          // bf16 element offset in the workspace
+  int32_t owners, r, rp;
+  int32_t pad_;
+  int64_t first_owner;      // prefix sum of owners
+};
+
+// fp32 factor -> [owners, 2rp] split bf16 (hi columns, then lo columns; columns >= r are zero)
+__global__ void __launch_bounds__(256) tc_convert_kernel(const ConvertJob* __restrict__ jobs, int n_jobs,
+                                                         int64_t total_owners, const float* __restrict__ state,
+                                                         uint16_t* __restrict__ work) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= total_owners) return;
+  int lo = 0, hi = n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (jobs[mid].first_owner <= gid) lo = mid; else hi = mid - 1;
+  }
+  const ConvertJob J = jobs[lo];
+  const int64_t owner = gid - J.first_owner;
+  const float* f = state + J.f32_off + J.own_stride * owner;
+  uint16_t* dst = work + J.dst_off + (int64_t)(2 * J.rp) * owner;
+  for (int p = 0; p < J.rp; p += 16) {
+    uint32_t h[8], l[8];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const int k = p + e;
+      const float x = k < J.r ? f[J.k_stride * k] : 0.f;
+      uint16_t a, b;
+      tc::split_bf16(x, a, b);
+      if (e & 1) { h[e >> 1] |= (uint32_t)a << 16; l[e >> 1] |= (uint32_t)b << 16; }
+      else { h[e >> 1] = a; l[e >> 1] = b; }
+    }
+    uint4* dh = reinterpret_cast<uint4*>(dst + p);
+    uint4* dl = reinterpret_cast<uint4*>(dst + J.rp + p);
+    dh[0] = make_uint4(h[0], h[1], h[2], h[3]);
+    dh[1] = make_uint4(h[4], h[5], h[6], h[7]);
+    dl[0] = make_uint4(l[0], l[1], l[2], l[3]);
+    dl[1] = make_uint4(l[4], l[5], l[6], l[7]);
+  }
 }
-void destroy_tensor_program(adapm_ctx*) {}
+
+}  // namespace
+
+// Host side of the tensor path, owned by the context.
+struct TcBlock {
+  int64_t id;                      // index into ctx->blocks
+  int32_t rp;
+  int64_t lc[3], rtc[3], gs[4];    // bf16 element offsets in the workspace
+};
+
+struct TcProgram {
+  std::vector<TcBlock> blk;
+  int64_t n_convert_owners = 0;
+  int smem_engine = 0, smem_apply = 0;
+  int engine_stage_bytes = 0, engine_stages = 0;
+  int apply_r_region = 0;
+  int n_sms = 148;
+  int final_set = 0;
+  // tensor maps: device table + pinned host staging, re-encoded when the buffers move
+  CUtensorMap* d_maps = nullptr;
+  CUtensorMap* h_maps = nullptr;
+  const void* enc_grads = nullptr;
+  const void* enc_work = nullptr;
+  cudaEvent_t maps_copied = nullptr;
+};
+
+bool tensor_path_block_ok(const adapm_hparams& hp, const adapm_block& b) {
+  if (hp.lowrank_path == ADAPM_PATH_SIMT) return false;
+  if (hp.grad_dtype != ADAPM_GRAD_BF16) return false;
+  if (b.mom_mode != ADAPM_MOM_LOWRANK) return false;
+  if (b.cols % 8 != 0 || b.rank > 128) return false;
+  return tc::encode_tiled_fn() != nullptr;
+}
+
+void destroy_tensor_program(adapm_ctx* c) {
+  TcProgram* p = c->tc;
+  if (!p) return;
+  if (p->d_maps) cudaFree(p->d_maps);
+  if (p->h_maps) cudaFreeHost(p->h_maps);
+  if (p->maps_copied) cudaEventDestroy(p->maps_copied);
+  delete p;
+  c->tc = nullptr;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// program construction
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+int round16(int x) { return (x + 15) / 16 * 16; }
+
+template <typename T>
+int64_t append_items(std::vector<unsigned char>& blob, const std::vector<T>& tab) {
+  const size_t off = (blob.size() + 15) / 16 * 16;
+  blob.resize(off + tab.size() * sizeof(T));
+  if (!tab.empty()) std::memcpy(blob.data() + off, tab.data(), tab.size() * sizeof(T));
+  return (int64_t)off;
+}
+
+tc::Seg make_seg(int map_a, int ax, int ay, int a_mode, int map_b, int bx, int by, int b_mode, int n, int k, int d_col,
+                 int first) {
+  tc::Seg s;
+  std::memset(&s, 0, sizeof(s));
+  s.map_a = map_a; s.map_b = map_b; s.ax = ax; s.ay = ay; s.bx = bx; s.by = by;
+  s.a_mode = (int16_t)a_mode; s.b_mode = (int16_t)b_mode;
+  s.n = (int16_t)n; s.nb_b = (int16_t)((n + 63) / 64); s.k = round16(k); s.d_col = (int16_t)d_col; s.first = (int16_t)first;
+  return s;
+}
+
+int item_cost(const tc::Item& it) {
+  int c = 0;
+  for (int s = 0; s < it.n_seg; ++s) c += (it.seg[s].k + 63) / 64;
+  return c + 2;   // the epilogue
+}
+
+void sort_by_cost(std::vector<tc::Item>& v) {
+  for (auto& it : v) it.cost = item_cost(it);
+  std::stable_sort(v.begin(), v.end(), [](const tc::Item& a, const tc::Item& b) { return a.cost > b.cost; });
+}
+
+}  // namespace
+
+int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const std::vector<double>& etas,
+                         int64_t& work_cursor) {
+  TcProgram* P = new TcProgram();
+  c->tc = P;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess)
+    P->n_sms = prop.multiProcessorCount;
+  const adapm_hparams& hp = c->hp;
+  const float b1 = hp.beta1, a1 = 1.f - hp.beta1;
+
+  // ---- workspace arrays (bf16), offsets counted in bf16 elements ------------------------------------
+  auto take = [&](int64_t bf16_elems) {
+    const int64_t off = work_cursor * 2;
+    work_cursor += round_up((bf16_elems + 1) / 2, kStateAlign);
+    return off;
+  };
+  int rp_max = 16;
+  for (int64_t id : tc_ids) {
+    const adapm_block& b = c->blocks[id];
+    TcBlock t;
+    t.id = id;
+    t.rp = round16(b.rank);
+    rp_max = std::max(rp_max, t.rp);
+    for (int s = 0; s < 3; ++s) t.lc[s] = take((int64_t)b.rows * 2 * t.rp);
+    for (int s = 0; s < 3; ++s) t.rtc[s] = take((int64_t)b.cols * 2 * t.rp);
+    for (int w = 0; w < 4; ++w) t.gs[w] = take((int64_t)2 * t.rp * t.rp);
+    P->blk.push_back(t);
+  }
+  const int nb_max = (2 * rp_max + 63) / 64;
+  P->engine_stage_bytes = tc::kStageABytes + tc::kBoxBytes * nb_max;
+  P->engine_stages = std::min(8, (224 * 1024) / P->engine_stage_bytes);
+  P->smem_engine = P->engine_stage_bytes * P->engine_stages + 1024;
+
+  auto& prog = c->program;
+
+  // ---- convert -------------------------------------------------------------------------------------------
+  {
+    std::vector<ConvertJob> jobs;
+    int64_t owners = 0;
+    for (const TcBlock& t : P->blk) {
+      const adapm_block& b = c->blocks[t.id];
+      ConvertJob j;
+      std::memset(&j, 0, sizeof(j));
+      j.r = b.rank; j.rp = t.rp;
+      j.f32_off = c->l_off[t.id]; j.own_stride = b.rank; j.k_stride = 1; j.owners = b.rows; j.dst_off = t.lc[0];
+      j.first_owner = owners; owners += j.owners; jobs.push_back(j);
+      j.f32_off = c->r_off[t.id]; j.own_stride = 1; j.k_stride = b.cols; j.owners = b.cols; j.dst_off = t.rtc[0];
+      j.first_owner = owners; owners += j.owners; jobs.push_back(j);
+    }
+    P->n_convert_owners = owners;
+    Launch L{LK_TC_CONVERT, append_items(c->h_tables, jobs), (int64_t)jobs.size(), (owners + 255) / 256};
+    L.aux0 = owners;
+    prog.push_back(L);
+  }
+
+  // ---- refit passes ----------------------------------------------------------------------------------------
+  int src = 0;
+  for (size_t pass = 0; pass < etas.size(); ++pass) {
+    const int dst = src == 1 ? 2 : 1;
+    const float coef = (float)etas[pass] * a1;
+    std::vector<tc::Item> grams, panels;
+    for (size_t bi = 0; bi < P->blk.size(); ++bi) {
+      const TcBlock& t = P->blk[bi];
+      const adapm_block& b = c->blocks[t.id];
+      const int m = b.rows, n = b.cols, r = b.rank, rp = t.rp;
+      const int mb = (int)bi * kMapsPerBlock;
+      const int mG = mb + MAP_G, mLs = mb + MAP_LC + src, mL0 = mb + MAP_LC, mRs = mb + MAP_RTC + src,
+                mR0 = mb + MAP_RTC;
+      // Gram items: dst[j][k] = coef * sum_x A[x][j] B[x][k], both operands taken MN-major from [x, 2rp] arrays
+      auto gram = [&](int map_a, int map_b, int kext, int which, float sc) {
+        tc::Item it;
+        std::memset(&it, 0, sizeof(it));
+        it.n_seg = 2;
+        it.seg[0] = make_seg(map_a, 0, 0, 1, map_b, 0, 0, 1, 2 * rp, kext, 0, 1);
+        it.seg[1] = make_seg(map_a, rp, 0, 1, map_b, 0, 0, 1, 2 * rp, kext, 2 * rp, 1);
+        it.epi = tc::EPI_GRAM; it.r = r; it.rp = rp; it.coef = sc;
+        it.dst_off = t.gs[which]; it.dst_ld = rp;
+        grams.push_back(it);
+      };
+      gram(mRs, mRs, n, 0, -1.f / a1);      // Bop1 = -(R R^T) / (1-b1)
+      gram(mRs, mR0, n, 1, b1 / a1);        // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
+      gram(mLs, mLs, m, 2, -1.f / a1);      // Bop3 = -(L^T L) / (1-b1)
+      gram(mLs, mL0, m, 3, b1 / a1);        // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
+
+      auto panel = [&](bool is_L, int p0) {
+        tc::Item it;
+        std::memset(&it, 0, sizeof(it));
+        const int mS = is_L ? mLs : mRs, m0 = is_L ? mL0 : mR0;
+        const int g1 = mb + MAP_GS + (is_L ? 0 : 2), g2 = g1 + 1;
+        if (is_L) it.seg[0] = make_seg(mG, 0, p0, 0, mRs, 0, 0, 1, 2 * rp, n, 0, 1);      // g R^T over the columns
+        else it.seg[0] = make_seg(mG, p0, 0, 1, mLs, 0, 0, 1, 2 * rp, m, 0, 1);            // g^T L over the rows
+        it.seg[1] = make_seg(mS, 0, p0, 0, g1, 0, 0, 0, 2 * rp, rp, 0, 0);
+        it.seg[2] = make_seg(mS, rp, p0, 0, g1, 0, 0, 0, 2 * rp, rp, 0, 0);
+        it.seg[3] = make_seg(m0, 0, p0, 0, g2, 0, 0, 0, 2 * rp, rp, 0, 0);
+        it.seg[4] = make_seg(m0, rp, p0, 0, g2, 0, 0, 0, 2 * rp, rp, 0, 0);
+        it.n_seg = 5;
+        it.epi = tc::EPI_FACTOR; it.r = r; it.rp = rp; it.coef = coef;
+        it.own0 = p0; it.own_count = is_L ? m : n;
+        it.f32_off = is_L ? c->l_off[t.id] : c->r_off[t.id];
+        it.own_stride = is_L ? r : 1; it.k_stride = is_L ? 1 : n;
+        it.dst_off = is_L ? t.lc[dst] : t.rtc[dst]; it.dst_ld = 2 * rp;
+        panels.push_back(it);
+      };
+      for (int p0 = 0; p0 < m; p0 += 128) panel(true, p0);
+      for (int p0 = 0; p0 < n; p0 += 128) panel(false, p0);
+    }
+    sort_by_cost(grams);
+    sort_by_cost(panels);
+    Launch G{LK_TC_GRAM, append_items(c->h_tables, grams), (int64_t)grams.size(),
+             std::min<int64_t>((int64_t)grams.size(), P->n_sms)};
+    G.aux0 = 4 * rp_max; G.aux1 = 8 * rp_max <= 512 ? 2 : 1;
+    prog.push_back(G);
+    Launch Q{LK_TC_PANEL, append_items(c->h_tables, panels), (int64_t)panels.size(),
+             std::min<int64_t>((int64_t)panels.size(), P->n_sms)};
+    Q.aux0 = 2 * rp_max; Q.aux1 = 2;
+    prog.push_back(Q);
+    src = dst;
+  }
+  P->final_set = src;
+
+  // ---- apply ---------------------------------------------------------------------------------------------------
+  {
+    std::vector<tc::ApplyItem> items;
+    int l_region = 0, r_region = 0;
+    for (size_t bi = 0; bi < P->blk.size(); ++bi) {
+      const TcBlock& t = P->blk[bi];
+      const adapm_block& b = c->blocks[t.id];
+      const int mb = (int)bi * kMapsPerBlock;
+      const int nbc = (2 * t.rp + 63) / 64;
+      const int nt = nbc <= 3 ? 128 : 64;
+      l_region = std::max(l_region, 2 * nbc * 2 * tc::kBoxBytes);
+      r_region = std::max(r_region, 2 * nbc * (nt / 64) * tc::kBoxBytes);
+      const int tiles = (b.cols + nt - 1) / nt;
+      const int runs = (tiles + 15) / 16;
+      for (int p0 = 0; p0 < b.rows; p0 += 128) {
+        for (int q = 0; q < runs; ++q) {
+          tc::ApplyItem a;
+          std::memset(&a, 0, sizeof(a));
+          a.off = b.offset; a.v_off = c->v_off[t.id]; a.rows = b.rows; a.cols = b.cols; a.r = b.rank; a.rp = t.rp;
+          a.map_l0 = mb + MAP_LC; a.map_l1 = mb + MAP_LC + P->final_set;
+          a.map_r0 = mb + MAP_RTC; a.map_r1 = mb + MAP_RTC + P->final_set;
+          a.row0 = p0;
+          a.tile0 = (int)((int64_t)tiles * q / runs);
+          a.n_tiles = (int)((int64_t)tiles * (q + 1) / runs) - a.tile0;
+          a.nt = nt; a.nbc = nbc; a.v_mode = b.v_mode;
+          a.v_group_rows = b.v_group_rows == 0 ? b.rows : b.v_group_rows;
+          a.lr_scale = b.lr_scale; a.wd = b.weight_decay;
+          items.push_back(a);
+        }
+      }
+    }
+    P->apply_r_region = l_region;
+    P->smem_apply = l_region + r_region + 1024;
+    Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
+             std::min<int64_t>((int64_t)items.size(), P->n_sms)};
+    prog.push_back(A);
+  }
+
+  // ---- tensor maps -------------------------------------------------------------------------------------------------
+  const size_t map_bytes = P->blk.size() * kMapsPerBlock * sizeof(CUtensorMap);
+  cudaError_t e = cudaMalloc((void**)&P->d_maps, map_bytes);
+  if (e == cudaSuccess) e = cudaMallocHost((void**)&P->h_maps, map_bytes);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&P->maps_copied, cudaEventDisableTiming);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::tc_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P->smem_engine);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::tc_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P->smem_apply);
+  if (e != cudaSuccess) {
+    set_cuda_error(e, "build_tensor_program");
+    return ADAPM_ECUDA;
+  }
+  return ADAPM_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// per-step work
+// ---------------------------------------------------------------------------------------------------
+
+// Tensor maps hold absolute addresses: (re)build them when the gradient or workspace buffer moved.
+// The copy to the device is asynchronous on `s`; only a second move while that copy is still in
+// flight waits for it (the staging buffer is reused).
+int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
+  TcProgram* P = c->tc;
+  if (!P || P->blk.empty()) return ADAPM_OK;
+  if (P->enc_grads == b.p[BASE_GRADS] && P->enc_work == b.p[BASE_WORK]) return ADAPM_OK;
+  if (P->enc_grads) ADAPM_CUDA(cudaEventSynchronize(P->maps_copied));
+  const char* grads = static_cast<const char*>(b.p[BASE_GRADS]);
+  const char* work = static_cast<const char*>(b.p[BASE_WORK]);
+  for (size_t bi = 0; bi < P->blk.size(); ++bi) {
+    const TcBlock& t = P->blk[bi];
+    const adapm_block& blk = c->blocks[t.id];
+    CUtensorMap* m = P->h_maps + bi * kMapsPerBlock;
+    const uint64_t rows = blk.rows, cols = blk.cols, rp = t.rp;
+    bool ok = tc::encode_bf16_matrix(&m[MAP_G], grads + blk.offset * 2, rows, cols, cols);
+    for (int q = 0; q < 3; ++q) {
+      ok = ok && tc::encode_bf16_matrix(&m[MAP_LC + q], work + t.lc[q] * 2, rows, 2 * rp, 2 * rp);
+      ok = ok && tc::encode_bf16_matrix(&m[MAP_RTC + q], work + t.rtc[q] * 2, cols, 2 * rp, 2 * rp);
+    }
+    for (int q = 0; q < 4; ++q) ok = ok && tc::encode_bf16_matrix(&m[MAP_GS + q], work + t.gs[q] * 2, 2 * rp, rp, rp);
+    if (!ok) {
+      set_error_text("cuTensorMapEncodeTiled failed for a low-rank block");
+      return ADAPM_ECUDA;
+    }
+  }
+  ADAPM_CUDA(cudaMemcpyAsync(P->d_maps, P->h_maps, P->blk.size() * kMapsPerBlock * sizeof(CUtensorMap),
+                             cudaMemcpyHostToDevice, s));
+  ADAPM_CUDA(cudaEventRecord(P->maps_copied, s));
+  P->enc_grads = b.p[BASE_GRADS];
+  P->enc_work = b.p[BASE_WORK];
+  return ADAPM_OK;
+}
+
+int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepScalars& sc, cudaStream_t s) {
+  TcProgram* P = c->tc;
+  if (!P) return ADAPM_EUNSUPPORTED;
+  const unsigned char* tab = c->d_tables + L.table_off;
+  if (L.grid <= 0) return ADAPM_OK;
+  switch (L.kind) {
+    case LK_TC_CONVERT:
+      tc_convert_kernel<<<(unsigned)L.grid, 256, 0, s>>>((const ConvertJob*)tab, (int)L.n_items, L.aux0,
+                                                        (const float*)b.p[BASE_STATE], (uint16_t*)b.p[BASE_WORK]);
+      break;
+    case LK_TC_GRAM:
+    case LK_TC_PANEL: {
+      tc::EngineArgs a;
+      a.items = (const tc::Item*)tab; a.n_items = (int32_t)L.n_items; a.maps = P->d_maps;
+      a.f32_base = (float*)b.p[BASE_STATE]; a.work_bf16 = (uint16_t*)b.p[BASE_WORK]; a.status = c->d_status;
+      a.stage_bytes = P->engine_stage_bytes; a.n_stages = P->engine_stages;
+      a.acc_cols = (int32_t)L.aux0; a.n_acc = (int32_t)L.aux1;
+      tc::tc_items_kernel<<<(unsigned)L.grid, tc::kEngineThreads, P->smem_engine, s>>>(a);
+      break;
+    }
+    case LK_TC_APPLY: {
+      tc::ApplyArgs a;
+      a.items = (const tc::ApplyItem*)tab; a.n_items = (int32_t)L.n_items; a.maps = P->d_maps;
+      a.params = (float*)b.p[BASE_PARAMS]; a.grads = (const uint16_t*)b.p[BASE_GRADS];
+      a.state = (float*)b.p[BASE_STATE]; a.status = c->d_status; a.sc = sc;
+      a.use_new = sc.c1 != 0.f ? 1 : 0;
+      a.r_region_off = P->apply_r_region;
+      tc::tc_apply_kernel<<<(unsigned)L.grid, tc::kApplyThreads, P->smem_apply, s>>>(a);
+      break;
+    }
+    default:
+      return ADAPM_EUNSUPPORTED;
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    set_cuda_error(e, "run_tensor_launch");
+    return ADAPM_ECUDA;
+  }
+  return ADAPM_OK;
+}
 
 }  // namespace adapm

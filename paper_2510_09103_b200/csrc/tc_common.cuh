@@ -1,0 +1,173 @@
+// Blackwell (sm_100a) building blocks of the tensor-core low-rank path: mbarriers with bounded
+// waits, TMA tile loads, tcgen05 MMA / TMEM wrappers and the shared-memory matrix descriptors.
+//
+// Every operand tile in shared memory is made of 8 KB boxes of 64 rows x 64 bf16 (128 bytes per
+// row) written by TMA with the 128-byte swizzle.  Two views of such boxes are used:
+//   K-major   rows are the M (or N) index, the 64 elements of a row run along K.  A 128-row operand
+//             is two boxes stacked (row pitch 128 B, 8-row groups 1024 B apart).
+//   MN-major  rows are the K index, the 64 elements of a row run along M (or N).  A 128-wide operand
+//             is two boxes side by side, 8 KB apart; 8-row K groups are 1024 B apart.
+// One tcgen05.mma of kind::f16 consumes K = 16: a 32-byte step inside the 128-byte row for a K-major
+// operand, two 8-row groups (2048 B) for an MN-major one.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace adapm {
+namespace tc {
+
+constexpr int kBoxRows = 64;
+constexpr int kBoxCols = 64;                       // bf16 elements: 128 bytes
+constexpr int kBoxBytes = kBoxRows * kBoxCols * 2; // 8192
+constexpr uint32_t kSpinLimit = 1u << 22;          // bounded waits: ~1 s with the back-off below
+
+// status bits a kernel may set when a bounded wait runs out
+enum : int32_t { ST_WAIT_FULL = 1, ST_WAIT_EMPTY = 2, ST_WAIT_TMEM_FULL = 4, ST_WAIT_TMEM_EMPTY = 8, ST_WAIT_DRAIN = 16 };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// ---- mbarrier ------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("{\n.reg .b64 st;\nmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Waits for the phase with the given parity to complete.  Gives up after kSpinLimit polls or as
+// soon as another thread of the CTA has given up (*abort != 0); then sets *abort, records `code` in
+// the device status word and returns false.  Callers leave their loops on false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
+                                          int32_t code) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 32) {
+      __nanosleep(it > 4096 ? 256 : 32);
+      if ((it & 255u) == 0 && *abort) return false;
+    }
+  }
+  *abort = 1;
+  atomicOr(status, code);
+  return false;
+}
+
+// ---- TMA -----------------------------------------------------------------------------------------
+// One 64 x 64 bf16 box at element coordinates (x, y) of a 2-D tensor map; x must be a multiple of 8.
+__device__ __forceinline__ void tma_load_box(void* smem_dst, const void* tmap, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// ---- tcgen05 -------------------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+               "r"(cols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]; issued by one thread.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The mbarrier gets one arrival when every MMA this thread issued before has completed.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+// 16 consecutive fp32 columns of this thread's TMEM lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+      "[%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- descriptors -----------------------------------------------------------------------------------
+// Instruction descriptor of kind::f16 with bf16 operands and fp32 accumulation, M = 128.
+__device__ __host__ __forceinline__ uint32_t make_idesc(int n, bool a_mn_major, bool b_mn_major, bool negate_a) {
+  uint32_t d = 0;
+  d |= 1u << 4;                          // accumulator format: fp32
+  d |= 1u << 7;                          // A format: bf16
+  d |= 1u << 10;                         // B format: bf16
+  d |= (negate_a ? 1u : 0u) << 13;
+  d |= (a_mn_major ? 1u : 0u) << 15;
+  d |= (b_mn_major ? 1u : 0u) << 16;
+  d |= (uint32_t)(n >> 3) << 17;
+  d |= (uint32_t)(128 >> 4) << 24;
+  return d;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (addresses and offsets in 16-byte units).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;                // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                // layout: 128-byte swizzle
+  return d;
+}
+// K-major operand whose rows start at `smem_addr`; k16 = which 16-wide K step inside the 64-wide box.
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t smem_addr, int k16) {
+  return make_smem_desc(smem_addr + 32u * (uint32_t)k16, 16, 1024);
+}
+// MN-major operand made of boxes 8 KB apart; k16 = which 16-row K step inside the 64-row box.
+__device__ __forceinline__ uint64_t desc_mn_major(uint32_t smem_addr, int k16) {
+  return make_smem_desc(smem_addr + 2048u * (uint32_t)k16, kBoxBytes, 1024);
+}
+
+// ---- split bf16 --------------------------------------------------------------------------------------
+// x ~ hi + lo with both parts bf16 (round to nearest even): the pair carries about 16 significant bits.
+__device__ __forceinline__ uint16_t f32_to_bf16_rn(float x) {
+  uint32_t u = __float_as_uint(x);
+  if ((u & 0x7F800000u) == 0x7F800000u) return (uint16_t)(u >> 16);   // inf / nan: truncate
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+__device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
+  hi = f32_to_bf16_rn(x);
+  lo = f32_to_bf16_rn(x - __uint_as_float((uint32_t)hi << 16));
+}
+
+}  // namespace tc
+}  // namespace adapm
