@@ -182,7 +182,10 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
       const int hw = I.nt / 2;                            // columns per thread per tile: 32 or 64
       const float lr_s = sc.lr * I.lr_scale;
       float v_row = 0.f;
-      if (row_ok && I.v_mode == ADAPM_V_BLOCKMEAN) v_row = a.state[I.v_off + row / I.v_group_rows];
+      const bool grouped = I.v_mode == ADAPM_V_BLOCKMEAN;
+      if (row_ok && grouped) v_row = a.state[I.v_off + row / I.v_group_rows];
+      // one denominator per row when v is a group scalar: m^c / (sqrt(v) + eps) becomes a multiplication
+      const float k_ratio = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
       const int64_t row_base = I.off + (int64_t)row * I.cols;
       for (int t = 0; t < I.n_tiles; ++t, ++j) {
         const int acc = j & 1;
@@ -230,12 +233,15 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
             for (int x = 0; x < 8; ++x) {
               const float g = gf[x];
               const float mc = sc.cg * g + sc.c0 * d[8 * u + x];
-              float v = v_row;
-              if (vp) {
-                v = sc.beta2 * vv[x] + (1.f - sc.beta2) * (g * g);
+              if (grouped) {
+                float ratio = mc * k_ratio;
+                ratio = ratio > sc.clip ? sc.clip : (ratio < -sc.clip ? -sc.clip : ratio);
+                w[x] = w[x] - lr_s * (ratio + I.wd * w[x]);
+              } else {
+                const float v = sc.beta2 * vv[x] + (1.f - sc.beta2) * (g * g);
                 vv[x] = v;
+                w[x] = adapm_param_update(w[x], mc, v, sc, lr_s, I.wd);
               }
-              w[x] = adapm_param_update(w[x], mc, v, sc, lr_s, I.wd);
             }
             if (vp) store8f(vp, vv);
             store8f(a.params + row_base + col + 8 * u, w);

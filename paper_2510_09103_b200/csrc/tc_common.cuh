@@ -20,7 +20,8 @@ namespace tc {
 constexpr int kBoxRows = 64;
 constexpr int kBoxCols = 64;                       // bf16 elements: 128 bytes
 constexpr int kBoxBytes = kBoxRows * kBoxCols * 2; // 8192
-constexpr uint32_t kSpinLimit = 1u << 22;          // bounded waits: ~1 s with the back-off below
+constexpr uint32_t kSpinLimit = 1u << 20;          // bounded waits: about a second of polling in all
+constexpr uint32_t kSuspendHintNs = 1000;          // a poll may park the thread this long before it reports failure
 
 // status bits a kernel may set when a bounded wait runs out
 enum : int32_t { ST_WAIT_FULL = 1, ST_WAIT_EMPTY = 2, ST_WAIT_TMEM_FULL = 4, ST_WAIT_TMEM_EMPTY = 8, ST_WAIT_DRAIN = 16 };
@@ -43,9 +44,9 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }

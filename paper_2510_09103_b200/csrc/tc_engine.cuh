@@ -112,7 +112,8 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
+    // Lane 0 waits for the stage and arms its barrier; lanes 0..5 then issue one box each.
+    {
       int stage = 0;
       uint32_t phase = 0;
       uint32_t issued = 0;
@@ -121,31 +122,33 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         const Item& I = a.items[it];
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const Seg S = I.seg[s];
-          const CUtensorMap* ma = a.maps + S.map_a;
-          const CUtensorMap* mb = a.maps + S.map_b;
           const int nch = seg_chunks(S);
+          // this lane's box: lanes 0,1 the A side, lanes 2.. the B side
+          const bool is_a = lane < 2;
+          const int h = is_a ? lane : lane - 2;
+          const bool active = lane < 2 + S.nb_b;
+          const CUtensorMap* map = a.maps + (is_a ? S.map_a : S.map_b);
+          const int mode = is_a ? S.a_mode : S.b_mode;
+          const int x0 = (is_a ? S.ax : S.bx) + (mode ? 64 * h : 0);
+          const int y0 = (is_a ? S.ay : S.by) + (mode ? 0 : 64 * h);
+          const int dx = mode ? 0 : 64, dy = mode ? 64 : 0;
+          const int soff = is_a ? h * kBoxBytes : kStageABytes + h * kBoxBytes;
           for (int c = 0; c < nch; ++c) {
-            if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
-            uint8_t* sa = stages + (size_t)stage * a.stage_bytes;
-            uint8_t* sb = sa + kStageABytes;
-            mbar_arrive_expect_tx(&sh.full[stage], (uint32_t)(2 + S.nb_b) * kBoxBytes);
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const int x = S.a_mode ? S.ax + 64 * h : S.ax + 64 * c;
-              const int y = S.a_mode ? S.ay + 64 * c : S.ay + 64 * h;
-              tma_load_box(sa + h * kBoxBytes, ma, x, y, &sh.full[stage]);
+            bool got = true;
+            if (lane == 0) {
+              got = mbar_wait(&sh.empty[stage], phase ^ 1u, abort, a.status, ST_WAIT_EMPTY);
+              if (got) mbar_arrive_expect_tx(&sh.full[stage], (uint32_t)(2 + S.nb_b) * kBoxBytes);
             }
-            for (int h = 0; h < S.nb_b; ++h) {
-              const int x = S.b_mode ? S.bx + 64 * h : S.bx + 64 * c;
-              const int y = S.b_mode ? S.by + 64 * c : S.by + 64 * h;
-              tma_load_box(sb + h * kBoxBytes, mb, x, y, &sh.full[stage]);
-            }
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (!got) { ok = false; break; }
+            if (active)
+              tma_load_box(stages + (size_t)stage * a.stage_bytes + soff, map, x0 + dx * c, y0 + dy * c, &sh.full[stage]);
             ++issued;
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
           }
         }
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         // leave no copy in flight: every stage that was filled must have landed before the CTA exits
         const int back = issued < (uint32_t)a.n_stages ? (int)issued : a.n_stages;
         for (int q = 0; q < back; ++q) {
@@ -203,35 +206,47 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       const Item& I = a.items[it];
       const int acc = j % a.n_acc;
       const uint32_t acc_phase = (uint32_t)(j / a.n_acc) & 1u;
-      // every lane polls, then the warp agrees: the tensor-memory loads below need all 32 lanes
-      const bool got = mbar_wait(&sh.tfull[acc], acc_phase, abort, a.status, ST_WAIT_TMEM_FULL);
-      if (!__all_sync(0xffffffffu, got)) break;
+      const int rp = I.rp, r = I.r;
+      // EPI_FACTOR: the old factor values of the first 16 columns are requested before the wait
+      const int owner = I.own0 + q;
+      const bool own_ok = I.epi == EPI_FACTOR && owner < I.own_count;
+      float* f = a.f32_base + I.f32_off + I.own_stride * owner;
+      float old[16] = {};
+      if (own_ok) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) old[e] = e < r ? f[I.k_stride * e] : 0.f;
+      }
+      // one lane per warp polls (fewer pollers on the barrier), then the warp agrees: the
+      // tensor-memory loads below need all 32 lanes
+      bool got = true;
+      if (lane == 0) got = mbar_wait(&sh.tfull[acc], acc_phase, abort, a.status, ST_WAIT_TMEM_FULL);
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!got) break;
       tc_fence_after();
       const uint32_t t0 = tmem_base + lane_addr + (uint32_t)(acc * a.acc_cols);
-      const int rp = I.rp, r = I.r;
       if (I.epi == EPI_FACTOR) {
-        const int owner = I.own0 + q;
-        const bool own_ok = owner < I.own_count;
-        float* f = a.f32_base + I.f32_off + I.own_stride * owner;
         uint16_t* dst = a.work_bf16 + I.dst_off + (int64_t)I.dst_ld * owner;
         for (int p = 0; p < rp; p += 16) {
-          float d0[16], d1[16];
+          float d0[16], d1[16], nxt[16];
           tmem_ld16(t0 + (uint32_t)p, d0);
           tmem_ld16(t0 + (uint32_t)(rp + p), d1);
+          if (own_ok && p + 16 < rp) {     // the next 16 old values travel while this piece is processed
+#pragma unroll
+            for (int e = 0; e < 16; ++e) nxt[e] = p + 16 + e < r ? f[I.k_stride * (p + 16 + e)] : 0.f;
+          }
           tmem_ld_wait();
           if (own_ok) {
             uint32_t hi[8], lo[8];
+            float x[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) x[e] = p + e < r ? old[e] + I.coef * (d0[e] + d1[e]) : 0.f;
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+              if (p + e < r) f[I.k_stride * (p + e)] = x[e];
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const int k = p + e;
-              float x = 0.f;
-              if (k < r) {
-                float* fp = f + I.k_stride * k;
-                x = *fp + I.coef * (d0[e] + d1[e]);
-                *fp = x;
-              }
               uint16_t h, l;
-              split_bf16(x, h, l);
+              split_bf16(x[e], h, l);
               if (e & 1) { hi[e >> 1] |= (uint32_t)h << 16; lo[e >> 1] |= (uint32_t)l << 16; }
               else { hi[e >> 1] = h; lo[e >> 1] = l; }
             }
@@ -241,6 +256,8 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             dh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
             dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) old[e] = nxt[e];
           }
         }
       } else if (I.epi == EPI_GRAM) {

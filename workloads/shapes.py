@@ -128,6 +128,16 @@ def get_workload(name: str, rank_override: int = 0) -> Workload:
     llama350m  24 layers, d=1024, 16 heads, SwiGLU 2736, vocab 32000; bf16 grads, 5% heavy rows.
     gpt2_1p5b  48 layers, d=1600, 25 heads, FFN 6400, vocab 50257, ctx 1024; bf16 Gaussian grads.
     """
+    layers = None
+    if "@" in name:                  # "gpt2_1p5b@4": the same shapes with 4 layers (small profiling captures)
+        name, _, n_l = name.partition("@")
+        layers = int(n_l)
+    if layers is not None:
+        if name != "gpt2_1p5b":
+            raise KeyError("a layer count can only be given for gpt2_1p5b")
+        w = Workload(f"{name}@{layers}", _gpt2(layers, 1600, 25, 6400, 50257, 1024), "bf16", "normal", steps=20)
+        w.rank_override = int(rank_override)
+        return w
     if name == "tiny":
         w = Workload(name, _gpt2(2, 256, 4, 1024, 4096, 2048), "f32", "normal", steps=10,
                      beta2=0.999)
