@@ -6,6 +6,7 @@
 //   convert   (L_{t-1}, R_{t-1}) fp32 -> split-bf16 arrays  Lc[0] = [L hi | L lo]  (rows x 2rp)
 //                                                           RTc[0] = [R^T hi | R^T lo] (cols x 2rp)
 //   K_eff times:  gram    four r x r products of the current iterate (tensor cores) -> Gs[0..3]
+//                         (each stored transposed, [rp, 2rp] = [hi | lo], the layout the engine's N side reads)
 //                 panel   row panels update L, column panels update R (tensor cores); fp32 factors
 //                         are updated in place in the state, their split copies go to the other of
 //                         the two iterate sets Lc[1|2], RTc[1|2]
@@ -26,8 +27,10 @@ void set_error_text(const char* text);   // ctx.cu
 
 namespace {
 
-constexpr int kMapsPerBlock = 11;   // g, Lc[3], RTc[3], Gs[4]
-enum { MAP_G = 0, MAP_LC = 1, MAP_RTC = 4, MAP_GS = 7 };
+// tensor maps of one block: g; Lc[3] and RTc[3] each as a plain matrix (A side) and as 64-column
+// chunks (N side); Gs[4] as chunks
+constexpr int kMapsPerBlock = 17;
+enum { MAP_G = 0, MAP_LC = 1, MAP_LC_N = 4, MAP_RTC = 7, MAP_RTC_N = 10, MAP_GS = 13 };
 
 struct ConvertJob {
   int64_t f32_off;          // float offset of the factor in state
@@ -87,7 +90,7 @@ struct TcProgram {
   int64_t n_convert_owners = 0;
   int smem_engine = 0, smem_apply = 0;
   int engine_stage_bytes = 0, engine_stages = 0;
-  int apply_r_region = 0;
+  int apply_r_region = 0, apply_r_stage = 0, apply_r_stages = 1, apply_turn_off = 0;
   int n_sms = 148;
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
@@ -131,19 +134,22 @@ int64_t append_items(std::vector<unsigned char>& blob, const std::vector<T>& tab
   return (int64_t)off;
 }
 
-tc::Seg make_seg(int map_a, int ax, int ay, int a_mode, int map_b, int bx, int by, int b_mode, int n, int k, int d_col,
-                 int first) {
+// A: 2-D map `map_a`, first box at (ax, ay), K along x (a_mode 0) or along y (a_mode 1).
+// B: chunked map `map_b` whose boxes are b_rows x (64 * nb_b), K rows starting at 0.
+tc::Seg make_seg(int map_a, int ax, int ay, int a_mode, int map_b, int b_rows, int n, int k, int d_col, int first) {
   tc::Seg s;
   std::memset(&s, 0, sizeof(s));
-  s.map_a = map_a; s.map_b = map_b; s.ax = ax; s.ay = ay; s.bx = bx; s.by = by;
-  s.a_mode = (int16_t)a_mode; s.b_mode = (int16_t)b_mode;
-  s.n = (int16_t)n; s.nb_b = (int16_t)((n + 63) / 64); s.k = round16(k); s.d_col = (int16_t)d_col; s.first = (int16_t)first;
+  const int nb_b = (n + 63) / 64;
+  s.map_a = map_a; s.map_b = map_b; s.ax = ax; s.ay = ay; s.by = 0;
+  s.a_mode = (int16_t)a_mode; s.n = (int16_t)n; s.k = round16(k); s.d_col = (int16_t)d_col; s.first = (int16_t)first;
+  s.b_lbo = 128u * (uint32_t)b_rows;
+  s.tx_bytes = (uint32_t)tc::kStageABytes + 128u * (uint32_t)b_rows * (uint32_t)nb_b;
   return s;
 }
 
 int item_cost(const tc::Item& it) {
   int c = 0;
-  for (int s = 0; s < it.n_seg; ++s) c += (it.seg[s].k + 63) / 64;
+  for (int s = 0; s < it.n_seg; ++s) c += (it.seg[s].k + tc::kStageK - 1) / tc::kStageK;
   return c + 2;   // the epilogue
 }
 
@@ -168,7 +174,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
   // ---- workspace arrays (bf16), offsets counted in bf16 elements ------------------------------------
   auto take = [&](int64_t bf16_elems) {
     const int64_t off = work_cursor * 2;
-    work_cursor += round_up((bf16_elems + 1) / 2, kStateAlign);
+    work_cursor += round_up((bf16_elems + 128 + 1) / 2, kStateAlign);   // +256 B: see encode_bf16_chunked
     return off;
   };
   int rp_max = 16;
@@ -185,7 +191,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
   }
   const int nb_max = (2 * rp_max + 63) / 64;
   P->engine_stage_bytes = tc::kStageABytes + tc::kBoxBytes * nb_max;
-  P->engine_stages = std::min(8, (224 * 1024) / P->engine_stage_bytes);
+  P->engine_stages = std::max(2, std::min(8, (224 * 1024) / P->engine_stage_bytes));
   P->smem_engine = P->engine_stage_bytes * P->engine_stages + 1024;
 
   auto& prog = c->program;
@@ -222,34 +228,35 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       const int m = b.rows, n = b.cols, r = b.rank, rp = t.rp;
       const int mb = (int)bi * kMapsPerBlock;
       const int mG = mb + MAP_G, mLs = mb + MAP_LC + src, mL0 = mb + MAP_LC, mRs = mb + MAP_RTC + src,
-                mR0 = mb + MAP_RTC;
-      // Gram items: dst[j][k] = coef * sum_x A[x][j] B[x][k], both operands taken MN-major from [x, 2rp] arrays
-      auto gram = [&](int map_a, int map_b, int kext, int which, float sc) {
+                mR0 = mb + MAP_RTC, mLsN = mb + MAP_LC_N + src, mRsN = mb + MAP_RTC_N + src;
+      // Gram item: dst[k][j] = coef * sum_x Y[x][k] X[x][j]; Y (the A side, read MN-major in two
+      // 128-column windows: the hi columns, then the lo columns) and X (the N side) are [x, 2rp] arrays
+      auto gram = [&](int map_y, int map_x_n, int kext, int which, float sc) {
         tc::Item it;
         std::memset(&it, 0, sizeof(it));
         it.n_seg = 2;
-        it.seg[0] = make_seg(map_a, 0, 0, 1, map_b, 0, 0, 1, 2 * rp, kext, 0, 1);
-        it.seg[1] = make_seg(map_a, rp, 0, 1, map_b, 0, 0, 1, 2 * rp, kext, 2 * rp, 1);
+        it.seg[0] = make_seg(map_y, 0, 0, 1, map_x_n, 128, 2 * rp, kext, 0, 1);
+        it.seg[1] = make_seg(map_y, rp, 0, 1, map_x_n, 128, 2 * rp, kext, 2 * rp, 1);
         it.epi = tc::EPI_GRAM; it.r = r; it.rp = rp; it.coef = sc;
-        it.dst_off = t.gs[which]; it.dst_ld = rp;
+        it.dst_off = t.gs[which]; it.dst_ld = 2 * rp;
         grams.push_back(it);
       };
-      gram(mRs, mRs, n, 0, -1.f / a1);      // Bop1 = -(R R^T) / (1-b1)
-      gram(mRs, mR0, n, 1, b1 / a1);        // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
-      gram(mLs, mLs, m, 2, -1.f / a1);      // Bop3 = -(L^T L) / (1-b1)
-      gram(mLs, mL0, m, 3, b1 / a1);        // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
+      gram(mRs, mRsN, n, 0, -1.f / a1);     // Bop1[j][k] = -(R R^T)[j][k] / (1-b1), stored as [k][j]
+      gram(mR0, mRsN, n, 1, b1 / a1);       // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
+      gram(mLs, mLsN, m, 2, -1.f / a1);     // Bop3[j][k] = -(L^T L)[j][k] / (1-b1)
+      gram(mL0, mLsN, m, 3, b1 / a1);       // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
 
       auto panel = [&](bool is_L, int p0) {
         tc::Item it;
         std::memset(&it, 0, sizeof(it));
         const int mS = is_L ? mLs : mRs, m0 = is_L ? mL0 : mR0;
         const int g1 = mb + MAP_GS + (is_L ? 0 : 2), g2 = g1 + 1;
-        if (is_L) it.seg[0] = make_seg(mG, 0, p0, 0, mRs, 0, 0, 1, 2 * rp, n, 0, 1);      // g R^T over the columns
-        else it.seg[0] = make_seg(mG, p0, 0, 1, mLs, 0, 0, 1, 2 * rp, m, 0, 1);            // g^T L over the rows
-        it.seg[1] = make_seg(mS, 0, p0, 0, g1, 0, 0, 0, 2 * rp, rp, 0, 0);
-        it.seg[2] = make_seg(mS, rp, p0, 0, g1, 0, 0, 0, 2 * rp, rp, 0, 0);
-        it.seg[3] = make_seg(m0, 0, p0, 0, g2, 0, 0, 0, 2 * rp, rp, 0, 0);
-        it.seg[4] = make_seg(m0, rp, p0, 0, g2, 0, 0, 0, 2 * rp, rp, 0, 0);
+        if (is_L) it.seg[0] = make_seg(mG, 0, p0, 0, mRsN, 128, 2 * rp, n, 0, 1);     // g R^T over the columns
+        else it.seg[0] = make_seg(mG, p0, 0, 1, mLsN, 128, 2 * rp, m, 0, 1);           // g^T L over the rows
+        it.seg[1] = make_seg(mS, 0, p0, 0, g1, rp, 2 * rp, rp, 0, 0);
+        it.seg[2] = make_seg(mS, rp, p0, 0, g1, rp, 2 * rp, rp, 0, 0);
+        it.seg[3] = make_seg(m0, 0, p0, 0, g2, rp, 2 * rp, rp, 0, 0);
+        it.seg[4] = make_seg(m0, rp, p0, 0, g2, rp, 2 * rp, rp, 0, 0);
         it.n_seg = 5;
         it.epi = tc::EPI_FACTOR; it.r = r; it.rp = rp; it.coef = coef;
         it.own0 = p0; it.own_count = is_L ? m : n;
@@ -278,16 +285,14 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
   // ---- apply ---------------------------------------------------------------------------------------------------
   {
     std::vector<tc::ApplyItem> items;
-    int l_region = 0, r_region = 0;
+    int nbc_max = 1;
     for (size_t bi = 0; bi < P->blk.size(); ++bi) {
       const TcBlock& t = P->blk[bi];
       const adapm_block& b = c->blocks[t.id];
       const int mb = (int)bi * kMapsPerBlock;
       const int nbc = (2 * t.rp + 63) / 64;
-      const int nt = nbc <= 3 ? 128 : 64;
-      l_region = std::max(l_region, 2 * nbc * 2 * tc::kBoxBytes);
-      r_region = std::max(r_region, 2 * nbc * (nt / 64) * tc::kBoxBytes);
-      const int tiles = (b.cols + nt - 1) / nt;
+      nbc_max = std::max(nbc_max, nbc);
+      const int tiles = (b.cols + tc::kApplyNT - 1) / tc::kApplyNT;
       const int runs = (tiles + 15) / 16;
       for (int p0 = 0; p0 < b.rows; p0 += 128) {
         for (int q = 0; q < runs; ++q) {
@@ -299,15 +304,22 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           a.row0 = p0;
           a.tile0 = (int)((int64_t)tiles * q / runs);
           a.n_tiles = (int)((int64_t)tiles * (q + 1) / runs) - a.tile0;
-          a.nt = nt; a.nbc = nbc; a.v_mode = b.v_mode;
+          a.nbc = nbc; a.v_mode = b.v_mode;
           a.v_group_rows = b.v_group_rows == 0 ? b.rows : b.v_group_rows;
           a.lr_scale = b.lr_scale; a.wd = b.weight_decay;
           items.push_back(a);
         }
       }
     }
+    // shared memory: both factor sets of the L panel, a ring of R^T tiles (one set each), the
+    // turn-around buffers of the eight epilogue warps
+    const int l_region = 2 * nbc_max * tc::kBoxBytes;
+    const int turn_bytes = 8 * tc::kStageFloats * 4;
+    P->apply_r_stage = nbc_max * tc::kBoxBytes;
+    P->apply_r_stages = std::max(1, std::min(4, (225 * 1024 - l_region - turn_bytes) / P->apply_r_stage));
     P->apply_r_region = l_region;
-    P->smem_apply = l_region + r_region + 1024;
+    P->apply_turn_off = l_region + P->apply_r_stages * P->apply_r_stage;
+    P->smem_apply = P->apply_turn_off + turn_bytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
              std::min<int64_t>((int64_t)items.size(), P->n_sms)};
     prog.push_back(A);
@@ -348,12 +360,16 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
     const adapm_block& blk = c->blocks[t.id];
     CUtensorMap* m = P->h_maps + bi * kMapsPerBlock;
     const uint64_t rows = blk.rows, cols = blk.cols, rp = t.rp;
+    const uint32_t nb = (uint32_t)((2 * rp + 63) / 64);
     bool ok = tc::encode_bf16_matrix(&m[MAP_G], grads + blk.offset * 2, rows, cols, cols);
     for (int q = 0; q < 3; ++q) {
       ok = ok && tc::encode_bf16_matrix(&m[MAP_LC + q], work + t.lc[q] * 2, rows, 2 * rp, 2 * rp);
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_LC_N + q], work + t.lc[q] * 2, rows, 2 * rp, nb, 128);
       ok = ok && tc::encode_bf16_matrix(&m[MAP_RTC + q], work + t.rtc[q] * 2, cols, 2 * rp, 2 * rp);
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_RTC_N + q], work + t.rtc[q] * 2, cols, 2 * rp, nb, 128);
     }
-    for (int q = 0; q < 4; ++q) ok = ok && tc::encode_bf16_matrix(&m[MAP_GS + q], work + t.gs[q] * 2, 2 * rp, rp, rp);
+    for (int q = 0; q < 4; ++q)
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_GS + q], work + t.gs[q] * 2, rp, 2 * rp, nb, (uint32_t)rp);
     if (!ok) {
       set_error_text("cuTensorMapEncodeTiled failed for a low-rank block");
       return ADAPM_ECUDA;
@@ -393,7 +409,8 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.params = (float*)b.p[BASE_PARAMS]; a.grads = (const uint16_t*)b.p[BASE_GRADS];
       a.state = (float*)b.p[BASE_STATE]; a.status = c->d_status; a.sc = sc;
       a.use_new = sc.c1 != 0.f ? 1 : 0;
-      a.r_region_off = P->apply_r_region;
+      a.r_region_off = P->apply_r_region; a.r_stage_bytes = P->apply_r_stage; a.n_rstages = P->apply_r_stages;
+      a.turn_off = P->apply_turn_off;
       tc::tc_apply_kernel<<<(unsigned)L.grid, tc::kApplyThreads, P->smem_apply, s>>>(a);
       break;
     }

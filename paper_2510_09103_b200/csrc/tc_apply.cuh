@@ -8,7 +8,10 @@
 // and L of the panel stay in shared memory for the whole run; per column tile the matching rows of
 // R0^T and R^T are loaded and the products hi*hi + hi*lo + lo*hi of both factor pairs are
 // accumulated into one accumulator (the new pair with a negated A operand), so the accumulator
-// holds D = L0 R0 - L R.  Eight epilogue warps then stream g and W through registers.
+// holds D = L0 R0 - L R.  Eight epilogue warps then stream g and W through registers: a thread reads
+// one accumulator row from tensor memory, the warp turns its 32 x 16 piece around through a small
+// shared-memory buffer so that four lanes share a row, and g / W are accessed as 64-byte row
+// segments (the next piece's g and W are requested while the current one is processed).
 // The m x n matrices m_t, r_t and m^c are never stored.
 #pragma once
 
@@ -22,15 +25,17 @@ namespace adapm {
 namespace tc {
 
 constexpr int kApplyThreads = 320;
+constexpr int kApplyNT = 128;              // columns per tile
+constexpr int kStagePitch = 20;            // floats per row of a warp's 32 x 16 turn-around buffer
+constexpr int kStageFloats = 32 * kStagePitch;
 
 struct ApplyItem {
   int64_t off;               // element offset of the block in params / grads
   int64_t v_off;             // float offset of v in state
   int32_t rows, cols, r, rp;
-  int32_t map_l0, map_l1, map_r0, map_r1;   // split factors: [rows, 2rp] and [cols, 2rp]
+  int32_t map_l0, map_l1, map_r0, map_r1;   // split factors: [rows, 2rp] and [cols, 2rp], boxes of 64 x 128
   int32_t row0;              // first row of the panel
-  int32_t tile0, n_tiles;    // column tiles [tile0, tile0 + n_tiles) of width nt
-  int32_t nt;                // 64 or 128
+  int32_t tile0, n_tiles;    // column tiles [tile0, tile0 + n_tiles) of 128 columns
   int32_t nbc;               // 64-wide boxes across the 2rp split columns
   int32_t v_mode, v_group_rows;
   float lr_scale, wd;
@@ -46,11 +51,14 @@ struct ApplyArgs {
   int32_t* status;
   StepScalars sc;
   int32_t use_new;           // 0: c1 == 0, the refitted factors are not needed
-  int32_t r_region_off;      // byte offset of the R tile region inside the dynamic shared memory
+  int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
+  int32_t r_stage_bytes;     // one ring stage: the R^T rows of one tile and one factor set
+  int32_t n_rstages;         // ring depth (1..4)
+  int32_t turn_off;          // byte offset of the turn-around buffers
 };
 
 struct __align__(8) ApplyShared {
-  uint64_t lfull, lempty, rfull, rempty, tfull[2], tempty[2];
+  uint64_t lfull, lempty, rfull[4], rempty[4], tfull[2], tempty[2];
   uint32_t tmem_base;
   int abort;
 };
@@ -66,7 +74,8 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
   const int n_sets = a.use_new ? 2 : 1;
 
   if (threadIdx.x == 0) {
-    mbar_init(&sh.lfull, 1); mbar_init(&sh.lempty, 1); mbar_init(&sh.rfull, 1); mbar_init(&sh.rempty, 1);
+    mbar_init(&sh.lfull, 1); mbar_init(&sh.lempty, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(&sh.rfull[i], 1); mbar_init(&sh.rempty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 256); }
     sh.abort = 0;
     mbar_fence_init();
@@ -83,84 +92,86 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      uint32_t item_phase = 0, tile_phase = 0;
+      uint32_t item_phase = 0, rphase = 0;
+      int rs = 0;
       bool ok = true;
-      bool l_pending = false, r_pending = false;
+      int l_loads = 0, r_loads = 0;
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
         const ApplyItem I = a.items[it];
-        const int rb_n = I.nt / 64;
         if (!mbar_wait(&sh.lempty, item_phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
-        mbar_arrive_expect_tx(&sh.lfull, (uint32_t)(n_sets * I.nbc * 2) * kBoxBytes);
+        mbar_arrive_expect_tx(&sh.lfull, (uint32_t)(n_sets * I.nbc) * kBoxBytes);
         for (int set = 0; set < n_sets; ++set) {
           const CUtensorMap* m = a.maps + (set ? I.map_l1 : I.map_l0);
           for (int bc = 0; bc < I.nbc; ++bc)
-            for (int rb = 0; rb < 2; ++rb)
-              tma_load_box(smem_l + (size_t)((set * I.nbc + bc) * 2 + rb) * kBoxBytes, m, 64 * bc, I.row0 + 64 * rb,
-                           &sh.lfull);
+            tma_load_box(smem_l + (size_t)(set * I.nbc + bc) * kBoxBytes, m, 64 * bc, I.row0, &sh.lfull);
         }
-        l_pending = true;
-        for (int t = 0; t < I.n_tiles; ++t) {
-          if (!mbar_wait(&sh.rempty, tile_phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
-          const int col0 = (I.tile0 + t) * I.nt;
-          mbar_arrive_expect_tx(&sh.rfull, (uint32_t)(n_sets * I.nbc * rb_n) * kBoxBytes);
+        ++l_loads;
+        for (int t = 0; t < I.n_tiles && ok; ++t) {
+          const int col0 = (I.tile0 + t) * kApplyNT;
           for (int set = 0; set < n_sets; ++set) {
+            if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
             const CUtensorMap* m = a.maps + (set ? I.map_r1 : I.map_r0);
-            for (int bc = 0; bc < I.nbc; ++bc)
-              for (int rb = 0; rb < rb_n; ++rb)
-                tma_load_box(smem_r + (size_t)((set * I.nbc + bc) * rb_n + rb) * kBoxBytes, m, 64 * bc,
-                             col0 + 64 * rb, &sh.rfull);
+            uint8_t* dst = smem_r + (size_t)rs * a.r_stage_bytes;
+            mbar_arrive_expect_tx(&sh.rfull[rs], (uint32_t)I.nbc * kBoxBytes);
+            for (int bc = 0; bc < I.nbc; ++bc) tma_load_box(dst + (size_t)bc * kBoxBytes, m, 64 * bc, col0, &sh.rfull[rs]);
+            ++r_loads;
+            if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
           }
-          r_pending = true;
-          tile_phase ^= 1u;
         }
         item_phase ^= 1u;
       }
       if (!ok) {   // let the copies already issued land before the CTA exits
-        if (l_pending)
-          for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&sh.lfull, item_phase ^ 1u) &&
-                                  !mbar_try_wait(&sh.lfull, item_phase); ++spin) __nanosleep(64);
-        if (r_pending)
-          for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&sh.rfull, tile_phase ^ 1u) &&
-                                  !mbar_try_wait(&sh.rfull, tile_phase); ++spin) __nanosleep(64);
+        if (l_loads)
+          for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&sh.lfull, (uint32_t)(l_loads - 1) & 1u); ++spin)
+            __nanosleep(64);
+        const int back = r_loads < a.n_rstages ? r_loads : a.n_rstages;
+        for (int q = 0; q < back; ++q) {
+          int st = rs - 1 - q;
+          uint32_t ph = rphase;
+          if (st < 0) { st += a.n_rstages; ph ^= 1u; }
+          for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&sh.rfull[st], ph); ++spin) __nanosleep(64);
+        }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      uint32_t item_phase = 0, tile_phase = 0;
+      uint32_t item_phase = 0, rphase = 0;
+      int rs = 0;
       int j = 0;   // running tile count of this CTA
       bool ok = true;
       const uint32_t l_base = smem_u32(smem_l), r_base = smem_u32(smem_r);
+      const uint32_t dhi = desc_hi();
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
         const ApplyItem I = a.items[it];
-        const int rb_n = I.nt / 64;
-        const int ks = I.rp / 16;     // 16-wide K steps per part
+        const int ks = I.rp >> 4;     // 16-wide K steps per part
         if (!mbar_wait(&sh.lfull, item_phase, abort, a.status, ST_WAIT_FULL)) break;
-        for (int t = 0; t < I.n_tiles; ++t, ++j) {
+        for (int t = 0; t < I.n_tiles && ok; ++t, ++j) {
           const int acc = j & 1;
           const uint32_t acc_phase = (uint32_t)(j >> 1) & 1u;
-          if (!mbar_wait(&sh.rfull, tile_phase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
           if (!mbar_wait(&sh.tempty[acc], acc_phase ^ 1u, abort, a.status, ST_WAIT_TMEM_EMPTY)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d = tmem_base + (uint32_t)(acc * I.nt);
+          const uint32_t d = tmem_base + (uint32_t)(acc * kApplyNT);
           uint32_t accumulate = 0;
           for (int set = 0; set < n_sets; ++set) {
-            const uint32_t idesc = make_idesc(I.nt, false, false, set == 1);
-            for (int pair = 0; pair < 3; ++pair) {
-              const int pa = pair == 2 ? 1 : 0, pb = pair == 1 ? 1 : 0;   // hi*hi, hi*lo, lo*hi
-              for (int s = 0; s < ks; ++s) {
-                const int ka = pa * ks + s, kb = pb * ks + s;
-                const uint64_t da = desc_k_major(l_base + (uint32_t)((set * I.nbc + (ka >> 2)) * 2) * kBoxBytes, ka & 3);
-                const uint64_t db =
-                    desc_k_major(r_base + (uint32_t)((set * I.nbc + (kb >> 2)) * rb_n) * kBoxBytes, kb & 3);
-                mma_bf16(d, da, db, idesc, accumulate);
-                accumulate = 1;
-              }
+            if (!mbar_wait(&sh.rfull[rs], rphase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t idesc = make_idesc(kApplyNT, false, false, set == 1);
+            const uint32_t la = desc_lo(l_base + (uint32_t)(set * I.nbc) * kBoxBytes, 16);
+            const uint32_t rb = desc_lo(r_base + (uint32_t)(rs * a.r_stage_bytes), 16);
+            // K step k of a [.., 2rp] operand: box k / 4 (16 KB apart), 32 bytes per step inside it
+            auto kstep = [](int k) { return (uint32_t)((k >> 2) * (kBoxBytes >> 4) + (k & 3) * 2); };
+            for (int s = 0; s < ks; ++s) {      // hi * hi
+              mma_bf16(d, desc_join(la + kstep(s), dhi), desc_join(rb + kstep(s), dhi), idesc, accumulate);
+              accumulate = 1;
             }
+            for (int s = 0; s < ks; ++s)        // hi * lo
+              mma_bf16(d, desc_join(la + kstep(s), dhi), desc_join(rb + kstep(ks + s), dhi), idesc, 1u);
+            for (int s = 0; s < ks; ++s)        // lo * hi
+              mma_bf16(d, desc_join(la + kstep(ks + s), dhi), desc_join(rb + kstep(s), dhi), idesc, 1u);
+            mma_commit(&sh.rempty[rs]);
+            if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
           }
-          mma_commit(&sh.rempty);
-          mma_commit(&sh.tfull[acc]);
-          tile_phase ^= 1u;
+          if (ok) mma_commit(&sh.tfull[acc]);
         }
         if (ok) mma_commit(&sh.lempty);
         item_phase ^= 1u;
@@ -169,88 +180,102 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
   } else {
     // ------------------------------------------------------------------ epilogue
     const int e = warp - 2;
-    const int q = 32 * (warp & 3) + lane;                 // accumulator row of this thread
-    const int half = e >> 2;                              // which half of the tile's columns
-    const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+    const int wq4 = warp & 3;                             // which 32 accumulator rows this warp may read
+    const int half = e >> 2;                              // which 64 columns of the tile
+    const uint32_t lane_addr = (uint32_t)(32 * wq4) << 16;
+    float* turn = reinterpret_cast<float*>(smem + a.turn_off) + e * kStageFloats;
     const StepScalars sc = a.sc;
+    const int rsub = lane >> 2;                           // after the turn: row rsub + 8 i, i = 0..3
+    const int csub = 4 * (lane & 3);                      // and four columns starting here
     int j = 0;
     bool ok = true;
     for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
       const ApplyItem I = a.items[it];
-      const int row = I.row0 + q;
-      const bool row_ok = row < I.rows;
-      const int hw = I.nt / 2;                            // columns per thread per tile: 32 or 64
-      const float lr_s = sc.lr * I.lr_scale;
-      float v_row = 0.f;
       const bool grouped = I.v_mode == ADAPM_V_BLOCKMEAN;
-      if (row_ok && grouped) v_row = a.state[I.v_off + row / I.v_group_rows];
-      // one denominator per row when v is a group scalar: m^c / (sqrt(v) + eps) becomes a multiplication
-      const float k_ratio = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
-      const int64_t row_base = I.off + (int64_t)row * I.cols;
-      for (int t = 0; t < I.n_tiles; ++t, ++j) {
-        const int acc = j & 1;
-        const uint32_t acc_phase = (uint32_t)(j >> 1) & 1u;
-        const int cb = (I.tile0 + t) * I.nt + half * hw;
-        const uint32_t t0 = tmem_base + lane_addr + (uint32_t)(acc * I.nt + half * hw);
-        bool waited = false;
-        for (int c0 = 0; c0 < hw; c0 += 32) {
-          // gradient and parameters of 32 columns, requested before the accumulator is needed
-          uint4 gq[4];
-          float4 wq[8];
-          const int col = cb + c0;
+      const float lr_s = sc.lr * I.lr_scale;
+      int64_t rbase[4];
+      bool rok[4];
+      float kr[4];   // one denominator per row when v is a group scalar: m^c / (sqrt(v) + eps) becomes a product
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const bool in = row_ok && col + 8 * u + 8 <= I.cols;
-            gq[u] = in ? __ldg(reinterpret_cast<const uint4*>(a.grads + row_base + col + 8 * u)) : make_uint4(0, 0, 0, 0);
-            wq[2 * u] = in ? *reinterpret_cast<const float4*>(a.params + row_base + col + 8 * u) : make_float4(0, 0, 0, 0);
-            wq[2 * u + 1] =
-                in ? *reinterpret_cast<const float4*>(a.params + row_base + col + 8 * u + 4) : make_float4(0, 0, 0, 0);
-          }
-          if (!waited) {
-            const bool got = mbar_wait(&sh.tfull[acc], acc_phase, abort, a.status, ST_WAIT_TMEM_FULL);
-            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-            tc_fence_after();
-            waited = true;
-          }
-          float d[32];
-          tmem_ld16(t0 + (uint32_t)c0, d);
-          tmem_ld16(t0 + (uint32_t)(c0 + 16), d + 16);
-          tmem_ld_wait();
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            if (!(row_ok && col + 8 * u + 8 <= I.cols)) continue;
-            float gf[8];
-            GradBF16::unpack(gq[u], gf);
-            float w[8] = {wq[2 * u].x, wq[2 * u].y, wq[2 * u].z, wq[2 * u].w,
-                          wq[2 * u + 1].x, wq[2 * u + 1].y, wq[2 * u + 1].z, wq[2 * u + 1].w};
-            float vv[8];
-            float* vp = nullptr;
-            if (I.v_mode == ADAPM_V_ELEMENT) {
-              vp = a.state + I.v_off + (int64_t)row * I.cols + col + 8 * u;
-              load8f(vp, vv);
-            }
-#pragma unroll
-            for (int x = 0; x < 8; ++x) {
-              const float g = gf[x];
-              const float mc = sc.cg * g + sc.c0 * d[8 * u + x];
-              if (grouped) {
-                float ratio = mc * k_ratio;
-                ratio = ratio > sc.clip ? sc.clip : (ratio < -sc.clip ? -sc.clip : ratio);
-                w[x] = w[x] - lr_s * (ratio + I.wd * w[x]);
-              } else {
-                const float v = sc.beta2 * vv[x] + (1.f - sc.beta2) * (g * g);
-                vv[x] = v;
-                w[x] = adapm_param_update(w[x], mc, v, sc, lr_s, I.wd);
-              }
-            }
-            if (vp) store8f(vp, vv);
-            store8f(a.params + row_base + col + 8 * u, w);
-          }
-        }
-        if (!ok) break;
-        tc_fence_before();
-        mbar_arrive(&sh.tempty[acc]);
+      for (int i = 0; i < 4; ++i) {
+        const int row = I.row0 + 32 * wq4 + rsub + 8 * i;
+        rok[i] = row < I.rows;
+        rbase[i] = I.off + (int64_t)row * I.cols;
+        const float v_row = (rok[i] && grouped) ? a.state[I.v_off + row / I.v_group_rows] : 0.f;
+        kr[i] = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
       }
+      const int n_pieces = I.n_tiles * 4;                 // pieces of 16 columns this warp handles
+      float4 wq[4], wn[4];
+      uint2 gq[4], gn[4];
+      auto piece_col = [&](int gi) { return (I.tile0 + (gi >> 2)) * kApplyNT + half * 64 + (gi & 3) * 16 + csub; };
+      auto request = [&](int gi, float4* w, uint2* g) {
+        const int col = piece_col(gi);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const bool in = rok[i] && col + 4 <= I.cols;
+          w[i] = in ? *reinterpret_cast<const float4*>(a.params + rbase[i] + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+          g[i] = in ? __ldg(reinterpret_cast<const uint2*>(a.grads + rbase[i] + col)) : make_uint2(0u, 0u);
+        }
+      };
+      request(0, wq, gq);
+      for (int gi = 0; gi < n_pieces; ++gi) {
+        const int jt = j + (gi >> 2), sub = gi & 3;
+        const int acc = jt & 1;
+        if (gi + 1 < n_pieces) request(gi + 1, wn, gn);
+        if (sub == 0) {
+          bool got = true;
+          if (lane == 0) got = mbar_wait(&sh.tfull[acc], (uint32_t)(jt >> 1) & 1u, abort, a.status, ST_WAIT_TMEM_FULL);
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) { ok = false; break; }
+          tc_fence_after();
+        }
+        float d[16];
+        tmem_ld16(tmem_base + lane_addr + (uint32_t)(acc * kApplyNT + half * 64 + sub * 16), d);
+        tmem_ld_wait();
+        float4* mine = reinterpret_cast<float4*>(turn + lane * kStagePitch);
+        mine[0] = make_float4(d[0], d[1], d[2], d[3]);
+        mine[1] = make_float4(d[4], d[5], d[6], d[7]);
+        mine[2] = make_float4(d[8], d[9], d[10], d[11]);
+        mine[3] = make_float4(d[12], d[13], d[14], d[15]);
+        __syncwarp();
+        const int col = piece_col(gi);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 dv = *reinterpret_cast<const float4*>(turn + (rsub + 8 * i) * kStagePitch + csub);
+          if (!(rok[i] && col + 4 <= I.cols)) continue;
+          const float dd[4] = {dv.x, dv.y, dv.z, dv.w};
+          const float gf[4] = {__uint_as_float(gq[i].x << 16), __uint_as_float(gq[i].x & 0xffff0000u),
+                               __uint_as_float(gq[i].y << 16), __uint_as_float(gq[i].y & 0xffff0000u)};
+          float w[4] = {wq[i].x, wq[i].y, wq[i].z, wq[i].w};
+          if (grouped) {
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              float ratio = (sc.cg * gf[x] + sc.c0 * dd[x]) * kr[i];
+              ratio = ratio > sc.clip ? sc.clip : (ratio < -sc.clip ? -sc.clip : ratio);
+              w[x] = w[x] - lr_s * (ratio + I.wd * w[x]);
+            }
+          } else {
+            float4* vp = reinterpret_cast<float4*>(a.state + I.v_off + (rbase[i] - I.off) + col);
+            const float4 vo = *vp;
+            float vv[4] = {vo.x, vo.y, vo.z, vo.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              vv[x] = sc.beta2 * vv[x] + (1.f - sc.beta2) * (gf[x] * gf[x]);
+              w[x] = adapm_param_update(w[x], sc.cg * gf[x] + sc.c0 * dd[x], vv[x], sc, lr_s, I.wd);
+            }
+            *vp = make_float4(vv[0], vv[1], vv[2], vv[3]);
+          }
+          *reinterpret_cast<float4*>(a.params + rbase[i] + col) = make_float4(w[0], w[1], w[2], w[3]);
+        }
+        __syncwarp();
+        if (sub == 3) {
+          tc_fence_before();
+          mbar_arrive(&sh.tempty[acc]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { wq[i] = wn[i]; gq[i] = gn[i]; }
+      }
+      j += I.n_tiles;
     }
   }
 

@@ -1,12 +1,12 @@
 // Blackwell (sm_100a) building blocks of the tensor-core low-rank path: mbarriers with bounded
 // waits, TMA tile loads, tcgen05 MMA / TMEM wrappers and the shared-memory matrix descriptors.
 //
-// Every operand tile in shared memory is made of 8 KB boxes of 64 rows x 64 bf16 (128 bytes per
+// Every operand tile in shared memory is made of boxes of up to 128 rows x 64 bf16 (128 bytes per
 // row) written by TMA with the 128-byte swizzle.  Two views of such boxes are used:
-//   K-major   rows are the M (or N) index, the 64 elements of a row run along K.  A 128-row operand
-//             is two boxes stacked (row pitch 128 B, 8-row groups 1024 B apart).
-//   MN-major  rows are the K index, the 64 elements of a row run along M (or N).  A 128-wide operand
-//             is two boxes side by side, 8 KB apart; 8-row K groups are 1024 B apart.
+//   K-major   rows are the M index, the 64 elements of a row run along K (8-row groups 1024 B
+//             apart); the next 64 of K are the next box.
+//   MN-major  rows are the K index, the 64 elements of a row run along M (or N).  A wider operand
+//             is several boxes side by side, one box size apart; 8-row K groups are 1024 B apart.
 // One tcgen05.mma of kind::f16 consumes K = 16: a 32-byte step inside the 128-byte row for a K-major
 // operand, two 8-row groups (2048 B) for an MN-major one.
 #pragma once
@@ -17,9 +17,9 @@
 namespace adapm {
 namespace tc {
 
-constexpr int kBoxRows = 64;
+constexpr int kBoxRows = 128;
 constexpr int kBoxCols = 64;                       // bf16 elements: 128 bytes
-constexpr int kBoxBytes = kBoxRows * kBoxCols * 2; // 8192
+constexpr int kBoxBytes = kBoxRows * kBoxCols * 2; // 16384
 constexpr uint32_t kSpinLimit = 1u << 20;          // bounded waits: about a second of polling in all
 constexpr uint32_t kSuspendHintNs = 1000;          // a poll may park the thread this long before it reports failure
 
@@ -69,12 +69,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 }
 
 // ---- TMA -----------------------------------------------------------------------------------------
-// One 64 x 64 bf16 box at element coordinates (x, y) of a 2-D tensor map; x must be a multiple of 8.
+// One box at element coordinates (x, y) of a 2-D tensor map; x must be a multiple of 8.
 __device__ __forceinline__ void tma_load_box(void* smem_dst, const void* tmap, int x, int y, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
           smem_u32(smem_dst)),
       "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// One box at (x, y, z) of a 3-D tensor map.
+__device__ __forceinline__ void tma_load_box3(void* smem_dst, const void* tmap, int x, int y, int z, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
       : "memory");
 }
 
@@ -148,13 +157,20 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
   d |= (uint64_t)2 << 61;                // layout: 128-byte swizzle
   return d;
 }
-// K-major operand whose rows start at `smem_addr`; k16 = which 16-wide K step inside the 64-wide box.
-__device__ __forceinline__ uint64_t desc_k_major(uint32_t smem_addr, int k16) {
-  return make_smem_desc(smem_addr + 32u * (uint32_t)k16, 16, 1024);
+// The same descriptor as two 32-bit halves, so that stepping through K only adds to the low half.
+// low: start address and leading byte offset; high: stride byte offset, version, swizzle mode.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+  return ((smem_addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }
-// MN-major operand made of boxes 8 KB apart; k16 = which 16-row K step inside the 64-row box.
-__device__ __forceinline__ uint64_t desc_mn_major(uint32_t smem_addr, int k16) {
-  return make_smem_desc(smem_addr + 2048u * (uint32_t)k16, kBoxBytes, 1024);
+__device__ __forceinline__ uint32_t desc_hi() { return (1024u >> 4) | (1u << 14) | (2u << 29); }
+__device__ __forceinline__ uint64_t desc_join(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
+// K-major operand (8-row groups 1024 B apart); k16 = which 16-wide K step inside the 64-wide box.
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t smem_addr, int k16) {
+  return desc_join(desc_lo(smem_addr + 32u * (uint32_t)k16, 16), desc_hi());
+}
+// MN-major operand made of boxes `lbo_bytes` apart; k16 = which 16-row K step inside the box.
+__device__ __forceinline__ uint64_t desc_mn_major(uint32_t smem_addr, int k16, uint32_t lbo_bytes) {
+  return desc_join(desc_lo(smem_addr + 2048u * (uint32_t)k16, lbo_bytes), desc_hi());
 }
 
 // ---- split bf16 --------------------------------------------------------------------------------------

@@ -8,7 +8,7 @@
 //   refit of R (column panel of 128 columns, the R update, computed transposed):
 //       D = g^T L + R^T Bop3^T + R0^T Bop4^T       Bop3 = -(L^T L)/(1-b1),  Bop4 = b1 (L^T L0)/(1-b1)
 //       R'^T = R^T + eta (1-b1) D
-//   Gram item: one of the r x r matrices above, scaled and stored as a split-bf16 B operand.
+//   Gram item: one of the r x r matrices above, scaled and stored (transposed) as a split-bf16 operand.
 //
 // fp32 factors are carried into the bf16 tensor cores as hi + lo pairs (two bf16 numbers whose sum
 // has ~16 significant bits); gradients are bf16 already and enter unchanged.  Operands with hi and
@@ -16,10 +16,16 @@
 // 16), so that used as the N side of an MMA the two parts land in two column ranges of the
 // accumulator, which the epilogue adds.
 //
-// Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 issues the MMAs,
-// warps 2-5 drain the accumulator.  With two accumulator buffers the epilogue of one item overlaps
-// the K-loops of the next.  Every wait is bounded; when one runs out the CTA records a status bit,
-// stops taking work and leaves through the common exit (which frees its tensor memory).
+// A stage of the shared-memory ring holds K = 128 of both operands:
+//   A  two boxes of 64 x 128 (32 KB): 128 rows x K (K along x) or K x 128 columns (K along y)
+//   B  one 3-D box: K rows x (64 x nb_b) columns of an [rows, 2rp] array, i.e. the N side read
+//      MN-major with its 64-column chunks one box apart
+// Warp roles (192 threads): warp 0 issues the three TMA loads of a stage, warp 1 issues its (up to)
+// eight MMAs, warps 2-5 drain the accumulator.  The two issuing threads run dependent scalar code, so
+// their per-stage instruction count is what bounds the rate; both loops are kept short.  With two
+// accumulator buffers the epilogue of one item overlaps the K-loops of the next.  Every wait is
+// bounded; when one runs out the CTA records a status bit, stops taking work and leaves through the
+// common exit (which frees its tensor memory).
 #pragma once
 
 #include <cuda.h>
@@ -30,18 +36,22 @@ namespace adapm {
 namespace tc {
 
 constexpr int kMaxSegs = 6;
-constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 128 x 64 bf16
+constexpr int kStageK = 128;
+constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 32 KB
 constexpr int kEngineThreads = 192;
 
 enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1, EPI_DUMP = 2 };
 
 struct Seg {
-  int32_t map_a, map_b;      // tensor-map indices
-  int32_t ax, ay, bx, by;    // element coordinates of the first box of each operand
-  int16_t a_mode, b_mode;    // 0: K runs along x (K-major), 1: K runs along y (MN-major)
-  int16_t nb_b;              // 64-wide boxes of B per chunk = ceil(n / 64)
-  int16_t n;                 // MMA N (multiple of 16, <= 256)
+  int32_t map_a;             // 2-D tensor map, box 64 x 128
+  int32_t map_b;             // 3-D tensor map (64, rows, chunks), box 64 x b_rows x nb_b
+  int32_t ax, ay;            // element coordinates of the first A box
+  int32_t by;                // first K row of B
   int32_t k;                 // K extent, multiple of 16
+  uint32_t b_lbo;            // bytes between the 64-column chunks of B in shared memory (= 128 * b_rows)
+  uint32_t tx_bytes;         // bytes one stage of this segment brings in
+  int16_t a_mode;            // 0: K runs along x (K-major A), 1: K runs along y (MN-major A)
+  int16_t n;                 // MMA N (multiple of 16, <= 256)
   int16_t d_col;             // accumulator column this segment starts at
   int16_t first;             // 1: its first MMA overwrites the accumulator
 };
@@ -54,7 +64,7 @@ struct Item {
   //   f32[own_stride * owner + k_stride * k] += coef * (D[q][k] + D[q][rp + k])        k < r
   //   dst[owner][k] = hi, dst[owner][rp + k] = lo                                      k < rp
   // EPI_GRAM: G[q][k] = coef * (D[q][k] + D[q][rp+k] + D[q][2rp+k] + D[q][3rp+k]);
-  //   dst[q][k] = hi, dst[rp + q][k] = lo                                              q, k < rp
+  //   dst[q][k] = hi, dst[q][rp + k] = lo                                              q, k < rp
   // EPI_DUMP: f32[q * n_dump + j] = D[q][j]                                            j < n_dump
   int32_t own0, own_count;   // first owner and number of owners of the whole matrix
   int32_t r, rp;
@@ -64,7 +74,7 @@ struct Item {
   int32_t dst_ld;            // its row pitch in elements
   int32_t n_dump;
   float coef;
-  int32_t cost;              // chunks, for scheduling
+  int32_t cost;              // stages, for scheduling
 };
 
 struct EngineArgs {
@@ -74,7 +84,7 @@ struct EngineArgs {
   float* f32_base;           // state buffer (or dump buffer)
   uint16_t* work_bf16;       // workspace viewed as bf16
   int32_t* status;
-  int32_t stage_bytes;       // kStageABytes + 8 KB * (largest nb_b)
+  int32_t stage_bytes;       // kStageABytes + 16 KB * (largest number of 64-column chunks of B)
   int32_t n_stages;
   int32_t acc_cols;          // tensor-memory columns per accumulator buffer
   int32_t n_acc;             // 1 or 2 accumulator buffers
@@ -86,7 +96,7 @@ struct __align__(8) EngineShared {
   int abort;
 };
 
-__device__ __forceinline__ int seg_chunks(const Seg& s) { return (s.k + kBoxCols - 1) / kBoxCols; }
+__device__ __forceinline__ int seg_stages(const Seg& s) { return (s.k + kStageK - 1) / kStageK; }
 
 __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs a) {
   extern __shared__ uint8_t dyn_smem[];
@@ -112,8 +122,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
-    // Lane 0 waits for the stage and arms its barrier; lanes 0..5 then issue one box each.
-    {
+    if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       uint32_t issued = 0;
@@ -122,33 +131,27 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         const Item& I = a.items[it];
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const Seg S = I.seg[s];
-          const int nch = seg_chunks(S);
-          // this lane's box: lanes 0,1 the A side, lanes 2.. the B side
-          const bool is_a = lane < 2;
-          const int h = is_a ? lane : lane - 2;
-          const bool active = lane < 2 + S.nb_b;
-          const CUtensorMap* map = a.maps + (is_a ? S.map_a : S.map_b);
-          const int mode = is_a ? S.a_mode : S.b_mode;
-          const int x0 = (is_a ? S.ax : S.bx) + (mode ? 64 * h : 0);
-          const int y0 = (is_a ? S.ay : S.by) + (mode ? 0 : 64 * h);
-          const int dx = mode ? 0 : 64, dy = mode ? 64 : 0;
-          const int soff = is_a ? h * kBoxBytes : kStageABytes + h * kBoxBytes;
-          for (int c = 0; c < nch; ++c) {
-            bool got = true;
-            if (lane == 0) {
-              got = mbar_wait(&sh.empty[stage], phase ^ 1u, abort, a.status, ST_WAIT_EMPTY);
-              if (got) mbar_arrive_expect_tx(&sh.full[stage], (uint32_t)(2 + S.nb_b) * kBoxBytes);
-            }
-            got = __shfl_sync(0xffffffffu, got, 0);
-            if (!got) { ok = false; break; }
-            if (active)
-              tma_load_box(stages + (size_t)stage * a.stage_bytes + soff, map, x0 + dx * c, y0 + dy * c, &sh.full[stage]);
+          const CUtensorMap* ma = a.maps + S.map_a;
+          const CUtensorMap* mb = a.maps + S.map_b;
+          const int nst = seg_stages(S);
+          // coordinates of the two A boxes and of the B box of the first stage, and their steps
+          int x0 = S.ax, y0 = S.ay, x1 = S.ax + 64, y1 = S.ay, yb = S.by;
+          const int dx = S.a_mode ? 0 : kStageK, dy = S.a_mode ? kStageK : 0;
+          for (int c = 0; c < nst; ++c) {
+            if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
+            uint8_t* sa = stages + stage * a.stage_bytes;
+            uint64_t* bar = &sh.full[stage];
+            mbar_arrive_expect_tx(bar, S.tx_bytes);
+            tma_load_box(sa, ma, x0, y0, bar);
+            tma_load_box(sa + kBoxBytes, ma, x1, y1, bar);
+            tma_load_box3(sa + kStageABytes, mb, 0, yb, 0, bar);
+            x0 += dx; x1 += dx; y0 += dy; y1 += dy; yb += kStageK;
             ++issued;
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
           }
         }
       }
-      if (!ok && lane == 0) {
+      if (!ok) {
         // leave no copy in flight: every stage that was filled must have landed before the CTA exits
         const int back = issued < (uint32_t)a.n_stages ? (int)issued : a.n_stages;
         for (int q = 0; q < back; ++q) {
@@ -166,6 +169,8 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       uint32_t phase = 0;
       bool ok = true;
       int j = 0;
+      const uint32_t stages_u32 = smem_u32(stages);
+      const uint32_t dhi = desc_hi();
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x, ++j) {
         const Item& I = a.items[it];
         const int acc = j % a.n_acc;
@@ -175,20 +180,28 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         const uint32_t d_base = tmem_base + (uint32_t)(acc * a.acc_cols);
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const Seg S = I.seg[s];
-          const uint32_t idesc = make_idesc(S.n, S.a_mode != 0, S.b_mode != 0, false);
-          const int nch = seg_chunks(S);
-          for (int c = 0; c < nch; ++c) {
+          const uint32_t idesc = make_idesc(S.n, S.a_mode != 0, true, false);
+          const uint32_t d = d_base + (uint32_t)S.d_col;
+          const int nst = seg_stages(S);
+          // per K step of 16, in 16-byte units: K along x walks 32 B inside a box and 16 KB to the
+          // next box; K along y walks 16 rows of 128 B
+          const uint32_t a_lbo = S.a_mode ? (uint32_t)kBoxBytes : 16u;
+          uint32_t accumulate = S.first ? 0u : 1u;
+          int k_left = S.k;
+          for (int c = 0; c < nst; ++c, k_left -= kStageK) {
             if (!mbar_wait(&sh.full[stage], phase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t sa = smem_u32(stages + (size_t)stage * a.stage_bytes);
-            const uint32_t sb = sa + kStageABytes;
-            int nk = (S.k - 64 * c + 15) / 16;
-            nk = nk > 4 ? 4 : nk;
-            for (int q = 0; q < nk; ++q) {
-              const uint64_t da = S.a_mode ? desc_mn_major(sa, q) : desc_k_major(sa, q);
-              const uint64_t db = S.b_mode ? desc_mn_major(sb, q) : desc_k_major(sb, q);
-              const uint32_t accumulate = (S.first && c == 0 && q == 0) ? 0u : 1u;
-              mma_bf16(d_base + (uint32_t)S.d_col, da, db, idesc, accumulate);
+            const uint32_t sa = stages_u32 + (uint32_t)(stage * a.stage_bytes);
+            const uint32_t alo = desc_lo(sa, a_lbo);
+            const uint32_t blo = desc_lo(sa + kStageABytes, S.b_lbo);
+            const int nk = k_left >= kStageK ? 8 : (k_left + 15) >> 4;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              if (q < nk) {
+                const uint32_t astep = S.a_mode ? (uint32_t)(q * 128) : (uint32_t)((q >> 2) * (kBoxBytes >> 4) + (q & 3) * 2);
+                mma_bf16(d, desc_join(alo + astep, dhi), desc_join(blo + (uint32_t)(q * 128), dhi), idesc, accumulate);
+                accumulate = 1u;
+              }
             }
             mma_commit(&sh.empty[stage]);
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
@@ -280,7 +293,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
               else { hi[e >> 1] = h; lo[e >> 1] = l; }
             }
             uint4* dh = reinterpret_cast<uint4*>(dst + (int64_t)I.dst_ld * q + p);
-            uint4* dl = reinterpret_cast<uint4*>(dst + (int64_t)I.dst_ld * (rp + q) + p);
+            uint4* dl = reinterpret_cast<uint4*>(dst + (int64_t)I.dst_ld * q + rp + p);
             dh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
             dh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
             dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
