@@ -218,7 +218,14 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   }
   if (!sblk.empty()) {
     const int64_t off = append_table(c->h_tables, sblk);
-    prog.push_back({LK_STREAM, off, (int64_t)sblk.size(), cta_cursor});
+    std::vector<int32_t> cta_blk((size_t)cta_cursor);       // CTA index -> entry of the block table
+    for (size_t i = 0; i < sblk.size(); ++i) {
+      const int64_t end = i + 1 < sblk.size() ? sblk[i + 1].first_cta : cta_cursor;
+      for (int64_t q = sblk[i].first_cta; q < end; ++q) cta_blk[(size_t)q] = (int32_t)i;
+    }
+    Launch SL{LK_STREAM, off, (int64_t)sblk.size(), cta_cursor};
+    SL.aux0 = append_table(c->h_tables, cta_blk);
+    prog.push_back(SL);
   }
 
   // ---- low-rank program --------------------------------------------------------------------------
@@ -470,7 +477,8 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
       case LK_REDUCE_FINAL:
         rc = launch_reduce_final((const ReduceJob*)tab, L.n_items, L.aux0, (float*)state, work, hp.beta2, s); break;
       case LK_STREAM:
-        rc = launch_stream((const StreamBlk*)tab, L.n_items, L.grid, b, sc, hp.grad_dtype, s); break;
+        rc = launch_stream((const StreamBlk*)tab, (const int32_t*)(c->d_tables + L.aux0), L.grid, b, sc, hp.grad_dtype, s);
+        break;
       case LK_GEMM:
         rc = launch_gemm((const GemmProb*)tab, L.n_items, L.grid, b, hp.grad_dtype, s); break;
       case LK_APPLY_SIMT:

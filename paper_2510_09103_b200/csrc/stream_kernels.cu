@@ -30,7 +30,8 @@ __device__ __forceinline__ float team_sum(float x, float* smem8) {
   return s;
 }
 
-template <typename GT, int TEAM>
+// One work unit.  HAS_M: the block keeps full momentum; HAS_V: v is per element.
+template <typename GT, int TEAM, bool HAS_M, bool HAS_V>
 __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float* __restrict__ params,
                                          const typename GT::elem* __restrict__ grads, float* __restrict__ state,
                                          const StepScalars& sc, float* smem8) {
@@ -53,7 +54,8 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
   }
   const typename GT::elem* g = grads + B.off + ustart;
   float* W = params + B.off + ustart;
-  float* M = (B.m_off >= 0) ? state + B.m_off + ustart : nullptr;
+  float* M = HAS_M ? state + B.m_off + ustart : nullptr;
+  float* V = HAS_V ? state + B.v_off + ustart : nullptr;
   const int nchunks = (ulen + kChunkElems - 1) / kChunkElems;
   const bool vec = B.vec_ok != 0;
 
@@ -70,10 +72,17 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
       } else {
         graw[c] = GT::load8_guarded(g + e0, ulen - e0);
       }
-      float f[8];
-      GT::unpack(graw[c], f);
+    }
+  }
+  if (B.v_mode == SV_GROUP_INLINE) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+    for (int c = 0; c < kTeamChunks; ++c) {
+      if (lane + c * TEAM < nchunks) {
+        float f[8];
+        GT::unpack(graw[c], f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+      }
     }
   }
 
@@ -95,85 +104,110 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
   } else if (B.v_mode == SV_GROUP_READY) {
     v_group = state[B.v_off + group];
   }
-  float* V = (B.v_mode == SV_ELEMENT) ? state + B.v_off + ustart : nullptr;
 
   // ---- phase 2: momentum, second moment, parameter write ------------------------------------
+  // Chunks are taken four at a time: all loads of a batch are issued before its first store, so the
+  // memory system sees them together instead of one round trip per chunk.
   const float lr_s = sc.lr * B.lr_scale;
   const float a1 = 1.f - sc.beta1, a2 = 1.f - sc.beta2;
+  // with a group scalar the division m^c / (sqrt(v) + eps) is one multiplication per element
+  const float k_ratio = sc.inv_bc1 / (sqrtf(v_group * sc.inv_bc2) + sc.eps);
+  constexpr int kBatch = ((HAS_M && HAS_V) || sizeof(typename GT::raw8) > 16) ? 2 : 4;
 #pragma unroll
-  for (int c = 0; c < kTeamChunks; ++c) {
-    const int idx = lane + c * TEAM;
-    if (idx < nchunks) {
-      const int e0 = idx * kChunkElems;
-      const bool full = vec && e0 + kChunkElems <= ulen;
-      const int nval = full ? 8 : (ulen - e0 < 8 ? ulen - e0 : 8);
-      float gf[8], w[8], m[8], v[8];
-      GT::unpack(graw[c], gf);
-      if (full) {
-        load8f(W + e0, w);
-        if (M) load8f(M + e0, m);
-        if (V) load8f(V + e0, v);
-      } else {
+  for (int c0 = 0; c0 < kTeamChunks; c0 += kBatch) {
+    float w[kBatch][8], m[kBatch][8], v[kBatch][8];
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int idx = lane + (c0 + b) * TEAM;
+      if (idx < nchunks) {
+        const int e0 = idx * kChunkElems;
+        if (vec && e0 + kChunkElems <= ulen) {
+          load8f(W + e0, w[b]);
+          if (HAS_M) load8f(M + e0, m[b]);
+          if (HAS_V) load8f(V + e0, v[b]);
+        } else {
+          const int nval = ulen - e0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const bool ok = i < nval;
+            w[b][i] = ok ? W[e0 + i] : 0.f;
+            if (HAS_M) m[b][i] = ok ? M[e0 + i] : 0.f;
+            if (HAS_V) v[b][i] = ok ? V[e0 + i] : 0.f;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < kBatch; ++b) {
+      const int idx = lane + (c0 + b) * TEAM;
+      if (idx < nchunks) {
+        const int e0 = idx * kChunkElems;
+        const bool full = vec && e0 + kChunkElems <= ulen;
+        float gf[8];
+        GT::unpack(graw[c0 + b], gf);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const bool ok = i < nval;
-          w[i] = ok ? W[e0 + i] : 0.f;
-          m[i] = (ok && M) ? M[e0 + i] : 0.f;
-          v[i] = (ok && V) ? V[e0 + i] : 0.f;
+          float mc = gf[i];
+          if (HAS_M) {
+            m[b][i] = sc.beta1 * m[b][i] + a1 * gf[i];
+            mc = m[b][i];
+          }
+          if (HAS_V) {
+            v[b][i] = sc.beta2 * v[b][i] + a2 * (gf[i] * gf[i]);
+            w[b][i] = adapm_param_update(w[b][i], mc, v[b][i], sc, lr_s, B.wd);
+          } else {
+            float ratio = mc * k_ratio;
+            ratio = ratio > sc.clip ? sc.clip : (ratio < -sc.clip ? -sc.clip : ratio);
+            w[b][i] = w[b][i] - lr_s * (ratio + B.wd * w[b][i]);
+          }
         }
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float mc = gf[i];
-        if (M) {
-          m[i] = sc.beta1 * m[i] + a1 * gf[i];
-          mc = m[i];
-        }
-        float vv = v_group;
-        if (V) {
-          v[i] = sc.beta2 * v[i] + a2 * (gf[i] * gf[i]);
-          vv = v[i];
-        }
-        w[i] = adapm_param_update(w[i], mc, vv, sc, lr_s, B.wd);
-      }
-      if (full) {
-        store8f(W + e0, w);
-        if (M) store8f(M + e0, m);
-        if (V) store8f(V + e0, v);
-      } else {
-        for (int i = 0; i < nval; ++i) {
-          W[e0 + i] = w[i];
-          if (M) M[e0 + i] = m[i];
-          if (V) V[e0 + i] = v[i];
+        if (full) {
+          store8f(W + e0, w[b]);
+          if (HAS_M) store8f(M + e0, m[b]);
+          if (HAS_V) store8f(V + e0, v[b]);
+        } else {
+          const int nval = ulen - e0 < 8 ? ulen - e0 : 8;
+          for (int i = 0; i < nval; ++i) {
+            W[e0 + i] = w[b][i];
+            if (HAS_M) M[e0 + i] = m[b][i];
+            if (HAS_V) V[e0 + i] = v[b][i];
+          }
         }
       }
     }
   }
 }
 
+template <typename GT, int TEAM>
+__device__ __forceinline__ void run_unit_any(const StreamBlk& B, int64_t unit, float* __restrict__ params,
+                                             const typename GT::elem* __restrict__ grads, float* __restrict__ state,
+                                             const StepScalars& sc, float* smem8) {
+  const bool has_m = B.m_off >= 0, has_v = B.v_mode == SV_ELEMENT;
+  if (has_m) {
+    if (has_v) run_unit<GT, TEAM, true, true>(B, unit, params, grads, state, sc, smem8);
+    else run_unit<GT, TEAM, true, false>(B, unit, params, grads, state, sc, smem8);
+  } else {
+    if (has_v) run_unit<GT, TEAM, false, true>(B, unit, params, grads, state, sc, smem8);
+    else run_unit<GT, TEAM, false, false>(B, unit, params, grads, state, sc, smem8);
+  }
+}
+
 template <typename GT>
-__global__ void __launch_bounds__(256) stream_update_kernel(const StreamBlk* __restrict__ tab, int n_blk,
-                                                            float* __restrict__ params,
-                                                            const typename GT::elem* __restrict__ grads,
-                                                            float* __restrict__ state, StepScalars sc) {
+__global__ void __launch_bounds__(256, 2) stream_update_kernel(const StreamBlk* __restrict__ tab,
+                                                               const int32_t* __restrict__ cta_blk,
+                                                               float* __restrict__ params,
+                                                               const typename GT::elem* __restrict__ grads,
+                                                               float* __restrict__ state, StepScalars sc) {
   __shared__ StreamBlk sB;
   __shared__ float smem8[12];
-  if (threadIdx.x == 0) {
-    int lo = 0, hi = n_blk - 1;            // last block with first_cta <= blockIdx.x
-    const int64_t me = blockIdx.x;
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (tab[mid].first_cta <= me) lo = mid; else hi = mid - 1;
-    }
-    sB = tab[lo];
-  }
+  if (threadIdx.x == 0) sB = tab[cta_blk[blockIdx.x]];   // which block this CTA works on
   __syncthreads();
   const int64_t cta_local = (int64_t)blockIdx.x - sB.first_cta;
   if (sB.team == 32) {
     const int64_t unit = cta_local * 8 + (threadIdx.x >> 5);
-    if (unit < sB.n_units) run_unit<GT, 32>(sB, unit, params, grads, state, sc, smem8);
+    if (unit < sB.n_units) run_unit_any<GT, 32>(sB, unit, params, grads, state, sc, smem8);
   } else {
-    run_unit<GT, 256>(sB, cta_local, params, grads, state, sc, smem8);
+    run_unit_any<GT, 256>(sB, cta_local, params, grads, state, sc, smem8);
   }
 }
 
@@ -295,15 +329,15 @@ __global__ void copy_f32_kernel(float4* __restrict__ dst, const float4* __restri
     }                                                \
   } while (0)
 
-int launch_stream(const StreamBlk* d_tab, int64_t n_blk, int64_t grid, const Bases& b, const StepScalars& sc,
-                  int grad_dtype, cudaStream_t s) {
+int launch_stream(const StreamBlk* d_tab, const int32_t* d_cta_blk, int64_t grid, const Bases& b,
+                  const StepScalars& sc, int grad_dtype, cudaStream_t s) {
   if (grid <= 0) return ADAPM_OK;
   if (grad_dtype == ADAPM_GRAD_BF16)
-    stream_update_kernel<GradBF16><<<(unsigned)grid, 256, 0, s>>>(d_tab, (int)n_blk, (float*)b.p[BASE_PARAMS],
+    stream_update_kernel<GradBF16><<<(unsigned)grid, 256, 0, s>>>(d_tab, d_cta_blk, (float*)b.p[BASE_PARAMS],
                                                                  (const uint16_t*)b.p[BASE_GRADS],
                                                                  (float*)b.p[BASE_STATE], sc);
   else
-    stream_update_kernel<GradF32><<<(unsigned)grid, 256, 0, s>>>(d_tab, (int)n_blk, (float*)b.p[BASE_PARAMS],
+    stream_update_kernel<GradF32><<<(unsigned)grid, 256, 0, s>>>(d_tab, d_cta_blk, (float*)b.p[BASE_PARAMS],
                                                                 (const float*)b.p[BASE_GRADS],
                                                                 (float*)b.p[BASE_STATE], sc);
   ADAPM_LAUNCH_CHECK();
