@@ -89,7 +89,19 @@ struct TcProgram {
   std::vector<TcBlock> blk;
   int64_t n_convert_owners = 0;
   int smem_engine = 0, smem_apply = 0;
-  int engine_stage_bytes = 0, engine_stages = 0;
+  int nb_max = 1;
+  // shared-memory plan of an engine launch: `wide` = stages with two A operands (no turn-around buffers)
+  struct EngineConfig { int a_bytes, stage_bytes, n_stages, turn_off, smem; };
+  EngineConfig engine_config(bool wide) const {
+    EngineConfig e;
+    const int turn = wide ? 0 : 8 * tc::kTurnFloats * 4;
+    e.a_bytes = (wide ? 2 : 1) * tc::kStageABytes;
+    e.stage_bytes = e.a_bytes + tc::kBoxBytes * nb_max;
+    e.n_stages = std::max(2, std::min(8, (224 * 1024 - turn) / e.stage_bytes));
+    e.turn_off = e.n_stages * e.stage_bytes;
+    e.smem = e.turn_off + turn + 1024;
+    return e;
+  }
   int apply_r_region = 0, apply_r_stage = 0, apply_r_stages = 1, apply_turn_off = 0;
   int n_sms = 148;
   int final_set = 0;
@@ -144,7 +156,14 @@ tc::Seg make_seg(int map_a, int ax, int ay, int a_mode, int map_b, int b_rows, i
   s.a_mode = (int16_t)a_mode; s.n = (int16_t)n; s.k = round16(k); s.d_col = (int16_t)d_col; s.first = (int16_t)first;
   s.b_lbo = 128u * (uint32_t)b_rows;
   s.tx_bytes = (uint32_t)tc::kStageABytes + 128u * (uint32_t)b_rows * (uint32_t)nb_b;
+  s.n_a = 1;
   return s;
+}
+
+// Adds a second A operand (same map and direction) that accumulates at column d_col2.
+void add_second_a(tc::Seg& s, int ax2, int ay2, int d_col2) {
+  s.n_a = 2; s.ax2 = ax2; s.ay2 = ay2; s.d_col2 = (int16_t)d_col2;
+  s.tx_bytes += (uint32_t)tc::kStageABytes;
 }
 
 int item_cost(const tc::Item& it) {
@@ -190,9 +209,15 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     P->blk.push_back(t);
   }
   const int nb_max = (2 * rp_max + 63) / 64;
-  P->engine_stage_bytes = tc::kStageABytes + tc::kBoxBytes * nb_max;
-  P->engine_stages = std::max(2, std::min(8, (224 * 1024) / P->engine_stage_bytes));
-  P->smem_engine = P->engine_stage_bytes * P->engine_stages + 1024;
+  // Gram items give every stage two A operands (the hi and the lo column window share each B box)
+  // when two such stages still fit.  Panel items keep one A operand: with two the accumulators fill
+  // the tensor memory, the epilogue can no longer overlap the next item, and that costs more than
+  // the saved loads bring (measured on the 1.5B set).
+  const bool two_a = 2 * (2 * tc::kStageABytes + tc::kBoxBytes * nb_max) <= 224 * 1024;
+  const bool pair_panels = false;
+  P->nb_max = nb_max;
+  P->smem_engine = 0;
+  for (int wide = 0; wide < 2; ++wide) P->smem_engine = std::max(P->smem_engine, P->engine_config(wide != 0).smem);
 
   auto& prog = c->program;
 
@@ -234,9 +259,15 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       auto gram = [&](int map_y, int map_x_n, int kext, int which, float sc) {
         tc::Item it;
         std::memset(&it, 0, sizeof(it));
-        it.n_seg = 2;
         it.seg[0] = make_seg(map_y, 0, 0, 1, map_x_n, 128, 2 * rp, kext, 0, 1);
-        it.seg[1] = make_seg(map_y, rp, 0, 1, map_x_n, 128, 2 * rp, kext, 2 * rp, 1);
+        if (two_a) {
+          it.n_seg = 1;
+          add_second_a(it.seg[0], rp, 0, 2 * rp);
+        } else {
+          it.n_seg = 2;
+          it.seg[1] = make_seg(map_y, rp, 0, 1, map_x_n, 128, 2 * rp, kext, 2 * rp, 1);
+        }
+        it.own1 = -1;
         it.epi = tc::EPI_GRAM; it.r = r; it.rp = rp; it.coef = sc;
         it.dst_off = t.gs[which]; it.dst_ld = 2 * rp;
         grams.push_back(it);
@@ -246,7 +277,8 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       gram(mLs, mLsN, m, 2, -1.f / a1);     // Bop3[j][k] = -(L^T L)[j][k] / (1-b1)
       gram(mL0, mLsN, m, 3, b1 / a1);       // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
 
-      auto panel = [&](bool is_L, int p0) {
+      // one item = one panel of 128 owners, or two adjacent panels that share every B box
+      auto panel = [&](bool is_L, int p0, bool pair) {
         tc::Item it;
         std::memset(&it, 0, sizeof(it));
         const int mS = is_L ? mLs : mRs, m0 = is_L ? mL0 : mR0;
@@ -258,6 +290,14 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         it.seg[3] = make_seg(m0, 0, p0, 0, g2, rp, 2 * rp, rp, 0, 0);
         it.seg[4] = make_seg(m0, rp, p0, 0, g2, rp, 2 * rp, rp, 0, 0);
         it.n_seg = 5;
+        it.own1 = -1;
+        if (pair) {
+          if (is_L) add_second_a(it.seg[0], 0, p0 + 128, 2 * rp);
+          else add_second_a(it.seg[0], p0 + 128, 0, 2 * rp);
+          for (int q = 1; q < 5; ++q) add_second_a(it.seg[q], it.seg[q].ax, p0 + 128, 2 * rp);
+          it.own1 = p0 + 128;
+          it.col2 = 2 * rp;
+        }
         it.epi = tc::EPI_FACTOR; it.r = r; it.rp = rp; it.coef = coef;
         it.own0 = p0; it.own_count = is_L ? m : n;
         it.f32_off = is_L ? c->l_off[t.id] : c->r_off[t.id];
@@ -265,18 +305,20 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         it.dst_off = is_L ? t.lc[dst] : t.rtc[dst]; it.dst_ld = 2 * rp;
         panels.push_back(it);
       };
-      for (int p0 = 0; p0 < m; p0 += 128) panel(true, p0);
-      for (int p0 = 0; p0 < n; p0 += 128) panel(false, p0);
+      const int step = pair_panels ? 256 : 128;
+      for (int p0 = 0; p0 < m; p0 += step) panel(true, p0, pair_panels && p0 + 128 < m);
+      for (int p0 = 0; p0 < n; p0 += step) panel(false, p0, pair_panels && p0 + 128 < n);
     }
     sort_by_cost(grams);
     sort_by_cost(panels);
     Launch G{LK_TC_GRAM, append_items(c->h_tables, grams), (int64_t)grams.size(),
              std::min<int64_t>((int64_t)grams.size(), P->n_sms)};
-    G.aux0 = 4 * rp_max; G.aux1 = 8 * rp_max <= 512 ? 2 : 1;
+    G.aux0 = 4 * rp_max; G.aux1 = 8 * rp_max <= 512 ? 2 : 1; G.aux2 = two_a ? 1 : 0;
     prog.push_back(G);
     Launch Q{LK_TC_PANEL, append_items(c->h_tables, panels), (int64_t)panels.size(),
              std::min<int64_t>((int64_t)panels.size(), P->n_sms)};
-    Q.aux0 = 2 * rp_max; Q.aux1 = 2;
+    Q.aux0 = (pair_panels ? 4 : 2) * rp_max; Q.aux1 = (pair_panels ? 8 : 4) * rp_max <= 512 ? 2 : 1;
+    Q.aux2 = pair_panels ? 1 : 0;
     prog.push_back(Q);
     src = dst;
   }
@@ -398,9 +440,10 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       tc::EngineArgs a;
       a.items = (const tc::Item*)tab; a.n_items = (int32_t)L.n_items; a.maps = P->d_maps;
       a.f32_base = (float*)b.p[BASE_STATE]; a.work_bf16 = (uint16_t*)b.p[BASE_WORK]; a.status = c->d_status;
-      a.stage_bytes = P->engine_stage_bytes; a.n_stages = P->engine_stages;
+      const TcProgram::EngineConfig e = P->engine_config(L.aux2 != 0);
+      a.stage_bytes = e.stage_bytes; a.n_stages = e.n_stages; a.a_bytes = e.a_bytes; a.turn_off = e.turn_off;
       a.acc_cols = (int32_t)L.aux0; a.n_acc = (int32_t)L.aux1;
-      tc::tc_items_kernel<<<(unsigned)L.grid, tc::kEngineThreads, P->smem_engine, s>>>(a);
+      tc::tc_items_kernel<<<(unsigned)L.grid, tc::kEngineThreads, e.smem, s>>>(a);
       break;
     }
     case LK_TC_APPLY: {

@@ -16,12 +16,16 @@
 // 16), so that used as the N side of an MMA the two parts land in two column ranges of the
 // accumulator, which the epilogue adds.
 //
-// A stage of the shared-memory ring holds K = 128 of both operands:
+// A stage of the shared-memory ring holds K = 128 of the operands:
 //   A  two boxes of 64 x 128 (32 KB): 128 rows x K (K along x) or K x 128 columns (K along y)
+//   A' optionally a second such operand (the next 128 rows / columns, or another column window):
+//      both are multiplied with the same B and fill two accumulators, which halves the bytes of B
+//      brought in per flop (the loads, not the tensor pipe, bound this kernel)
 //   B  one 3-D box: K rows x (64 x nb_b) columns of an [rows, 2rp] array, i.e. the N side read
 //      MN-major with its 64-column chunks one box apart
-// Warp roles (192 threads): warp 0 issues the three TMA loads of a stage, warp 1 issues its (up to)
-// eight MMAs, warps 2-5 drain the accumulator.  The two issuing threads run dependent scalar code, so
+// Warp roles (320 threads): warp 0 issues the TMA loads of a stage, warp 1 issues its (up to)
+// sixteen MMAs, warps 2-5 drain the first accumulator and warps 6-9 the second.  The two issuing
+// threads run dependent scalar code, so
 // their per-stage instruction count is what bounds the rate; both loops are kept short.  With two
 // accumulator buffers the epilogue of one item overlaps the K-loops of the next.  Every wait is
 // bounded; when one runs out the CTA records a status bit, stops taking work and leaves through the
@@ -38,7 +42,9 @@ namespace tc {
 constexpr int kMaxSegs = 6;
 constexpr int kStageK = 128;
 constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 32 KB
-constexpr int kEngineThreads = 192;
+constexpr int kEngineThreads = 320;
+constexpr int kTurnPitch = 20;                   // floats per row of a warp's 32 x 16 turn-around buffer
+constexpr int kTurnFloats = 32 * kTurnPitch;
 
 enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1, EPI_DUMP = 2 };
 
@@ -54,6 +60,9 @@ struct Seg {
   int16_t n;                 // MMA N (multiple of 16, <= 256)
   int16_t d_col;             // accumulator column this segment starts at
   int16_t first;             // 1: its first MMA overwrites the accumulator
+  int16_t n_a;               // 1, or 2: a second A operand at (ax2, ay2) accumulates at column d_col2
+  int16_t d_col2;
+  int32_t ax2, ay2;
 };
 
 struct Item {
@@ -67,6 +76,8 @@ struct Item {
   //   dst[q][k] = hi, dst[q][rp + k] = lo                                              q, k < rp
   // EPI_DUMP: f32[q * n_dump + j] = D[q][j]                                            j < n_dump
   int32_t own0, own_count;   // first owner and number of owners of the whole matrix
+  int32_t own1;              // EPI_FACTOR: first owner of the second accumulator (columns from col2), or -1
+  int32_t col2;
   int32_t r, rp;
   int64_t f32_off;           // float offset in the state buffer (EPI_DUMP: in the dump buffer)
   int64_t own_stride, k_stride;
@@ -84,7 +95,9 @@ struct EngineArgs {
   float* f32_base;           // state buffer (or dump buffer)
   uint16_t* work_bf16;       // workspace viewed as bf16
   int32_t* status;
-  int32_t stage_bytes;       // kStageABytes + 16 KB * (largest number of 64-column chunks of B)
+  int32_t stage_bytes;       // a_bytes + 16 KB * (largest number of 64-column chunks of B)
+  int32_t a_bytes;           // kStageABytes, or twice that when segments with two A operands occur
+  int32_t turn_off;          // byte offset (from the first stage) of the eight turn-around buffers of EPI_FACTOR
   int32_t n_stages;
   int32_t acc_cols;          // tensor-memory columns per accumulator buffer
   int32_t n_acc;             // 1 or 2 accumulator buffers
@@ -107,7 +120,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 8; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 256); }
     sh.abort = 0;
     mbar_fence_init();
   }
@@ -135,7 +148,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           const CUtensorMap* mb = a.maps + S.map_b;
           const int nst = seg_stages(S);
           // coordinates of the two A boxes and of the B box of the first stage, and their steps
-          int x0 = S.ax, y0 = S.ay, x1 = S.ax + 64, y1 = S.ay, yb = S.by;
+          int x0 = S.ax, y0 = S.ay, x2 = S.ax2, y2 = S.ay2, yb = S.by;
           const int dx = S.a_mode ? 0 : kStageK, dy = S.a_mode ? kStageK : 0;
           for (int c = 0; c < nst; ++c) {
             if (!mbar_wait(&sh.empty[stage], phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
@@ -143,9 +156,13 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             uint64_t* bar = &sh.full[stage];
             mbar_arrive_expect_tx(bar, S.tx_bytes);
             tma_load_box(sa, ma, x0, y0, bar);
-            tma_load_box(sa + kBoxBytes, ma, x1, y1, bar);
-            tma_load_box3(sa + kStageABytes, mb, 0, yb, 0, bar);
-            x0 += dx; x1 += dx; y0 += dy; y1 += dy; yb += kStageK;
+            tma_load_box(sa + kBoxBytes, ma, x0 + 64, y0, bar);
+            if (S.n_a == 2) {
+              tma_load_box(sa + kStageABytes, ma, x2, y2, bar);
+              tma_load_box(sa + kStageABytes + kBoxBytes, ma, x2 + 64, y2, bar);
+            }
+            tma_load_box3(sa + a.a_bytes, mb, 0, yb, 0, bar);
+            x0 += dx; y0 += dy; x2 += dx; y2 += dy; yb += kStageK;
             ++issued;
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
           }
@@ -181,7 +198,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const Seg S = I.seg[s];
           const uint32_t idesc = make_idesc(S.n, S.a_mode != 0, true, false);
-          const uint32_t d = d_base + (uint32_t)S.d_col;
+          const uint32_t d = d_base + (uint32_t)S.d_col, d2 = d_base + (uint32_t)S.d_col2;
           const int nst = seg_stages(S);
           // per K step of 16, in 16-byte units: K along x walks 32 B inside a box and 16 KB to the
           // next box; K along y walks 16 rows of 128 B
@@ -193,13 +210,16 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             tc_fence_after();
             const uint32_t sa = stages_u32 + (uint32_t)(stage * a.stage_bytes);
             const uint32_t alo = desc_lo(sa, a_lbo);
-            const uint32_t blo = desc_lo(sa + kStageABytes, S.b_lbo);
+            const uint32_t alo2 = desc_lo(sa + kStageABytes, a_lbo);
+            const uint32_t blo = desc_lo(sa + (uint32_t)a.a_bytes, S.b_lbo);
             const int nk = k_left >= kStageK ? 8 : (k_left + 15) >> 4;
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
               if (q < nk) {
                 const uint32_t astep = S.a_mode ? (uint32_t)(q * 128) : (uint32_t)((q >> 2) * (kBoxBytes >> 4) + (q & 3) * 2);
-                mma_bf16(d, desc_join(alo + astep, dhi), desc_join(blo + (uint32_t)(q * 128), dhi), idesc, accumulate);
+                const uint64_t bd = desc_join(blo + (uint32_t)(q * 128), dhi);
+                mma_bf16(d, desc_join(alo + astep, dhi), bd, idesc, accumulate);
+                if (S.n_a == 2) mma_bf16(d2, desc_join(alo2 + astep, dhi), bd, idesc, accumulate);
                 accumulate = 1u;
               }
             }
@@ -214,21 +234,42 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
     // ------------------------------------------------------------------ epilogue
     const int q = 32 * (warp & 3) + lane;               // accumulator row (= TMEM lane) of this thread
     const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+    const bool second = warp >= 6;                      // this warp drains the second accumulator
     int j = 0;
     for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++j) {
       const Item& I = a.items[it];
       const int acc = j % a.n_acc;
       const uint32_t acc_phase = (uint32_t)(j / a.n_acc) & 1u;
       const int rp = I.rp, r = I.r;
-      // EPI_FACTOR: the old factor values of the first 16 columns are requested before the wait
-      const int owner = I.own0 + q;
-      const bool own_ok = I.epi == EPI_FACTOR && owner < I.own_count;
-      float* f = a.f32_base + I.f32_off + I.own_stride * owner;
-      float old[16] = {};
-      if (own_ok) {
+      // EPI_FACTOR works in a "turned" layout: a thread reads its accumulator row from tensor memory,
+      // the warp passes each 32 x 16 piece through a small shared-memory buffer, and then four lanes
+      // share a row (lane -> rows rsub + 8 i, columns csub .. csub + 3), so that factor rows are read
+      // and written as 64-byte runs instead of one row per lane.
+      const bool has_work = !second || (I.epi == EPI_FACTOR && I.own1 >= 0);
+      const bool factor = I.epi == EPI_FACTOR && has_work;
+      const int own_base = (second ? I.own1 : I.own0) + 32 * (warp & 3);
+      const int rsub = lane >> 2, csub = 4 * (lane & 3);
+      float* fbase = a.f32_base + I.f32_off;
+      // float4 path: the four values of a lane are adjacent in memory and 16-byte aligned
+      const bool vec4 = I.k_stride == 1 && (I.own_stride & 3) == 0 && (r & 3) == 0 && (I.f32_off & 3) == 0;
+      float old[4][4];
+      auto fetch_old = [&](int p, float (*o)[4]) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) old[e] = e < r ? f[I.k_stride * e] : 0.f;
-      }
+        for (int i = 0; i < 4; ++i) {
+          const int owner = own_base + rsub + 8 * i;
+          const int k = p + csub;
+          const bool row_ok = owner < I.own_count;
+          const float* fp = fbase + I.own_stride * owner + I.k_stride * k;
+          if (vec4) {
+            const float4 v = (row_ok && k < r) ? *reinterpret_cast<const float4*>(fp) : make_float4(0.f, 0.f, 0.f, 0.f);
+            o[i][0] = v.x; o[i][1] = v.y; o[i][2] = v.z; o[i][3] = v.w;
+          } else {
+#pragma unroll
+            for (int x = 0; x < 4; ++x) o[i][x] = (row_ok && k + x < r) ? fp[I.k_stride * x] : 0.f;
+          }
+        }
+      };
+      if (factor) fetch_old(0, old);     // requested before the wait
       // one lane per warp polls (fewer pollers on the barrier), then the warp agrees: the
       // tensor-memory loads below need all 32 lanes
       bool got = true;
@@ -236,42 +277,54 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       got = __shfl_sync(0xffffffffu, got, 0);
       if (!got) break;
       tc_fence_after();
-      const uint32_t t0 = tmem_base + lane_addr + (uint32_t)(acc * a.acc_cols);
-      if (I.epi == EPI_FACTOR) {
-        uint16_t* dst = a.work_bf16 + I.dst_off + (int64_t)I.dst_ld * owner;
+      const uint32_t t0 = tmem_base + lane_addr + (uint32_t)(acc * a.acc_cols + (second ? I.col2 : 0));
+      if (!has_work) {
+        // nothing to drain for this warp; it still takes part in the hand-back below
+      } else if (I.epi == EPI_FACTOR) {
+        float* turn = reinterpret_cast<float*>(stages + a.turn_off) + (warp - 2) * kTurnFloats;
+        uint16_t* dst = a.work_bf16 + I.dst_off;
         for (int p = 0; p < rp; p += 16) {
-          float d0[16], d1[16], nxt[16];
+          float d0[16], d1[16], nxt[4][4];
           tmem_ld16(t0 + (uint32_t)p, d0);
           tmem_ld16(t0 + (uint32_t)(rp + p), d1);
-          if (own_ok && p + 16 < rp) {     // the next 16 old values travel while this piece is processed
-#pragma unroll
-            for (int e = 0; e < 16; ++e) nxt[e] = p + 16 + e < r ? f[I.k_stride * (p + 16 + e)] : 0.f;
-          }
+          if (p + 16 < rp) fetch_old(p + 16, nxt);   // the next old values travel while this piece is processed
           tmem_ld_wait();
-          if (own_ok) {
-            uint32_t hi[8], lo[8];
-            float x[16];
+          float4* mine = reinterpret_cast<float4*>(turn + lane * kTurnPitch);
+          mine[0] = make_float4(d0[0] + d1[0], d0[1] + d1[1], d0[2] + d1[2], d0[3] + d1[3]);
+          mine[1] = make_float4(d0[4] + d1[4], d0[5] + d1[5], d0[6] + d1[6], d0[7] + d1[7]);
+          mine[2] = make_float4(d0[8] + d1[8], d0[9] + d1[9], d0[10] + d1[10], d0[11] + d1[11]);
+          mine[3] = make_float4(d0[12] + d1[12], d0[13] + d1[13], d0[14] + d1[14], d0[15] + d1[15]);
+          __syncwarp();
 #pragma unroll
-            for (int e = 0; e < 16; ++e) x[e] = p + e < r ? old[e] + I.coef * (d0[e] + d1[e]) : 0.f;
+          for (int i = 0; i < 4; ++i) {
+            const float4 sv = *reinterpret_cast<const float4*>(turn + (rsub + 8 * i) * kTurnPitch + csub);
+            const int owner = own_base + rsub + 8 * i;
+            if (owner >= I.own_count) continue;
+            const int k = p + csub;
+            const float sd[4] = {sv.x, sv.y, sv.z, sv.w};
+            float x[4];
 #pragma unroll
-            for (int e = 0; e < 16; ++e)
-              if (p + e < r) f[I.k_stride * (p + e)] = x[e];
+            for (int e = 0; e < 4; ++e) x[e] = k + e < r ? old[i][e] + I.coef * sd[e] : 0.f;
+            float* fp = fbase + I.own_stride * owner + I.k_stride * k;
+            if (vec4) {
+              if (k < r) *reinterpret_cast<float4*>(fp) = make_float4(x[0], x[1], x[2], x[3]);
+            } else {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              uint16_t h, l;
-              split_bf16(x[e], h, l);
-              if (e & 1) { hi[e >> 1] |= (uint32_t)h << 16; lo[e >> 1] |= (uint32_t)l << 16; }
-              else { hi[e >> 1] = h; lo[e >> 1] = l; }
+              for (int e = 0; e < 4; ++e)
+                if (k + e < r) fp[I.k_stride * e] = x[e];
             }
-            uint4* dh = reinterpret_cast<uint4*>(dst + p);
-            uint4* dl = reinterpret_cast<uint4*>(dst + rp + p);
-            dh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            dh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-            dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-            dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+            uint16_t h[4], l[4];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) old[e] = nxt[e];
+            for (int e = 0; e < 4; ++e) split_bf16(x[e], h[e], l[e]);
+            uint16_t* drow = dst + (int64_t)I.dst_ld * owner + k;
+            *reinterpret_cast<uint2*>(drow) = make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+            *reinterpret_cast<uint2*>(drow + rp) = make_uint2((uint32_t)l[0] | ((uint32_t)l[1] << 16), (uint32_t)l[2] | ((uint32_t)l[3] << 16));
           }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) old[i][e] = nxt[i][e];
         }
       } else if (I.epi == EPI_GRAM) {
         uint16_t* dst = a.work_bf16 + I.dst_off;
