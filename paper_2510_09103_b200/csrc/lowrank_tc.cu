@@ -90,16 +90,14 @@ struct TcProgram {
   int64_t n_convert_owners = 0;
   int smem_engine = 0, smem_apply = 0;
   int nb_max = 1;
-  // shared-memory plan of an engine launch: `wide` = stages with two A operands (no turn-around buffers)
-  struct EngineConfig { int a_bytes, stage_bytes, n_stages, turn_off, smem; };
+  // shared-memory plan of an engine launch: `wide` = stages with two A operands
+  struct EngineConfig { int a_bytes, stage_bytes, n_stages, smem; };
   EngineConfig engine_config(bool wide) const {
     EngineConfig e;
-    const int turn = wide ? 0 : 8 * tc::kTurnFloats * 4;
     e.a_bytes = (wide ? 2 : 1) * tc::kStageABytes;
     e.stage_bytes = e.a_bytes + tc::kBoxBytes * nb_max;
-    e.n_stages = std::max(2, std::min(8, (224 * 1024 - turn) / e.stage_bytes));
-    e.turn_off = e.n_stages * e.stage_bytes;
-    e.smem = e.turn_off + turn + 1024;
+    e.n_stages = std::max(2, std::min(8, (224 * 1024) / e.stage_bytes));
+    e.smem = e.n_stages * e.stage_bytes + 1024;
     return e;
   }
   int apply_r_region = 0, apply_r_stage = 0, apply_r_stages = 1, apply_turn_off = 0;
@@ -209,15 +207,16 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     P->blk.push_back(t);
   }
   const int nb_max = (2 * rp_max + 63) / 64;
-  // Gram items give every stage two A operands (the hi and the lo column window share each B box)
-  // when two such stages still fit.  Panel items keep one A operand: with two the accumulators fill
-  // the tensor memory, the epilogue can no longer overlap the next item, and that costs more than
-  // the saved loads bring (measured on the 1.5B set).
+  // Every stage gets two A operands when two such stages still fit: Gram items read the hi and the
+  // lo column window of their A side against the same B boxes, panel items take two adjacent panels
+  // of a block.  Besides halving the B bytes per flop, consecutive MMAs then alternate between two
+  // accumulators instead of forming one dependent chain, which nearly doubles the issue rate.
   const bool two_a = 2 * (2 * tc::kStageABytes + tc::kBoxBytes * nb_max) <= 224 * 1024;
-  const bool pair_panels = false;
+  const bool pair_panels = two_a;
   P->nb_max = nb_max;
   P->smem_engine = 0;
-  for (int wide = 0; wide < 2; ++wide) P->smem_engine = std::max(P->smem_engine, P->engine_config(wide != 0).smem);
+  P->smem_engine = P->engine_config(false).smem;
+  if (two_a) P->smem_engine = std::max(P->smem_engine, P->engine_config(true).smem);
 
   auto& prog = c->program;
 
@@ -441,7 +440,7 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.items = (const tc::Item*)tab; a.n_items = (int32_t)L.n_items; a.maps = P->d_maps;
       a.f32_base = (float*)b.p[BASE_STATE]; a.work_bf16 = (uint16_t*)b.p[BASE_WORK]; a.status = c->d_status;
       const TcProgram::EngineConfig e = P->engine_config(L.aux2 != 0);
-      a.stage_bytes = e.stage_bytes; a.n_stages = e.n_stages; a.a_bytes = e.a_bytes; a.turn_off = e.turn_off;
+      a.stage_bytes = e.stage_bytes; a.n_stages = e.n_stages; a.a_bytes = e.a_bytes;
       a.acc_cols = (int32_t)L.aux0; a.n_acc = (int32_t)L.aux1;
       tc::tc_items_kernel<<<(unsigned)L.grid, tc::kEngineThreads, e.smem, s>>>(a);
       break;

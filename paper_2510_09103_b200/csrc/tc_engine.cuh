@@ -43,8 +43,6 @@ constexpr int kMaxSegs = 6;
 constexpr int kStageK = 128;
 constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 32 KB
 constexpr int kEngineThreads = 320;
-constexpr int kTurnPitch = 20;                   // floats per row of a warp's 32 x 16 turn-around buffer
-constexpr int kTurnFloats = 32 * kTurnPitch;
 
 enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1, EPI_DUMP = 2 };
 
@@ -97,7 +95,6 @@ struct EngineArgs {
   int32_t* status;
   int32_t stage_bytes;       // a_bytes + 16 KB * (largest number of 64-column chunks of B)
   int32_t a_bytes;           // kStageABytes, or twice that when segments with two A operands occur
-  int32_t turn_off;          // byte offset (from the first stage) of the eight turn-around buffers of EPI_FACTOR
   int32_t n_stages;
   int32_t acc_cols;          // tensor-memory columns per accumulator buffer
   int32_t n_acc;             // 1 or 2 accumulator buffers
@@ -242,22 +239,22 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       const uint32_t acc_phase = (uint32_t)(j / a.n_acc) & 1u;
       const int rp = I.rp, r = I.r;
       // EPI_FACTOR works in a "turned" layout: a thread reads its accumulator row from tensor memory,
-      // the warp passes each 32 x 16 piece through a small shared-memory buffer, and then four lanes
-      // share a row (lane -> rows rsub + 8 i, columns csub .. csub + 3), so that factor rows are read
-      // and written as 64-byte runs instead of one row per lane.
+      // then every quad of lanes transposes its 4 x 16 piece with shuffles, after which lane c of the
+      // quad holds columns 4c .. 4c+3 of the quad's four rows.  Factor rows are then read and written
+      // as 64-byte runs instead of one row per lane.  The old factor values of the first kPre pieces
+      // are requested before the accumulator is waited for.
       const bool has_work = !second || (I.epi == EPI_FACTOR && I.own1 >= 0);
       const bool factor = I.epi == EPI_FACTOR && has_work;
-      const int own_base = (second ? I.own1 : I.own0) + 32 * (warp & 3);
-      const int rsub = lane >> 2, csub = 4 * (lane & 3);
+      const int qc = lane & 3;
+      const int own_quad = (second ? I.own1 : I.own0) + 32 * (warp & 3) + (lane & ~3);
       float* fbase = a.f32_base + I.f32_off;
       // float4 path: the four values of a lane are adjacent in memory and 16-byte aligned
       const bool vec4 = I.k_stride == 1 && (I.own_stride & 3) == 0 && (r & 3) == 0 && (I.f32_off & 3) == 0;
-      float old[4][4];
       auto fetch_old = [&](int p, float (*o)[4]) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const int owner = own_base + rsub + 8 * i;
-          const int k = p + csub;
+          const int owner = own_quad + i;      // quad row i, this lane's four columns of it
+          const int k = p + 4 * qc;
           const bool row_ok = owner < I.own_count;
           const float* fp = fbase + I.own_stride * owner + I.k_stride * k;
           if (vec4) {
@@ -269,7 +266,13 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           }
         }
       };
-      if (factor) fetch_old(0, old);     // requested before the wait
+      constexpr int kPre = 6;            // pieces of 16 columns whose old values are fetched up front (rp <= 96)
+      float old[kPre][4][4];
+      if (factor) {
+#pragma unroll
+        for (int pi = 0; pi < kPre; ++pi)
+          if (16 * pi < rp) fetch_old(16 * pi, old[pi]);
+      }
       // one lane per warp polls (fewer pollers on the barrier), then the warp agrees: the
       // tensor-memory loads below need all 32 lanes
       bool got = true;
@@ -281,30 +284,57 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       if (!has_work) {
         // nothing to drain for this warp; it still takes part in the hand-back below
       } else if (I.epi == EPI_FACTOR) {
-        float* turn = reinterpret_cast<float*>(stages + a.turn_off) + (warp - 2) * kTurnFloats;
         uint16_t* dst = a.work_bf16 + I.dst_off;
-        for (int p = 0; p < rp; p += 16) {
-          float d0[16], d1[16], nxt[4][4];
+        // one piece: accumulator columns [p, p+16) of this thread's row, old values in `o`
+        auto piece = [&](int p, float (*o)[4]) {
+          float d0[16], d1[16];
           tmem_ld16(t0 + (uint32_t)p, d0);
           tmem_ld16(t0 + (uint32_t)(rp + p), d1);
-          if (p + 16 < rp) fetch_old(p + 16, nxt);   // the next old values travel while this piece is processed
           tmem_ld_wait();
-          float4* mine = reinterpret_cast<float4*>(turn + lane * kTurnPitch);
-          mine[0] = make_float4(d0[0] + d1[0], d0[1] + d1[1], d0[2] + d1[2], d0[3] + d1[3]);
-          mine[1] = make_float4(d0[4] + d1[4], d0[5] + d1[5], d0[6] + d1[6], d0[7] + d1[7]);
-          mine[2] = make_float4(d0[8] + d1[8], d0[9] + d1[9], d0[10] + d1[10], d0[11] + d1[11]);
-          mine[3] = make_float4(d0[12] + d1[12], d0[13] + d1[13], d0[14] + d1[14], d0[15] + d1[15]);
-          __syncwarp();
+          float v[4][4];                 // v[j] = columns 4j .. 4j+3 of this thread's row
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[j][e] = d0[4 * j + e] + d1[4 * j + e];
+          // quad transpose, round 1 (partner lane ^ 2): keep the half of the columns this lane's
+          // final column group lies in, hand over the other half
+          const bool up = (qc & 2) != 0, odd = (qc & 1) != 0;
+          float k0[4], k1[4], g0[4], g1[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            k0[e] = up ? v[2][e] : v[0][e];
+            k1[e] = up ? v[3][e] : v[1][e];
+            const float s0 = up ? v[0][e] : v[2][e], s1 = up ? v[1][e] : v[3][e];
+            g0[e] = __shfl_xor_sync(0xffffffffu, s0, 2);
+            g1[e] = __shfl_xor_sync(0xffffffffu, s1, 2);
+          }
+          // round 2 (partner lane ^ 1): keep this lane's column group of the two rows held so far,
+          // hand over the neighbour's; t[0..3] then belong to quad rows qc, qc^2, qc^1, qc^3
+          float t[4][4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            t[0][e] = odd ? k1[e] : k0[e];
+            t[1][e] = odd ? g1[e] : g0[e];
+            const float s0 = odd ? k0[e] : k1[e], s1 = odd ? g0[e] : g1[e];
+            t[2][e] = __shfl_xor_sync(0xffffffffu, s0, 1);
+            t[3][e] = __shfl_xor_sync(0xffffffffu, s1, 1);
+          }
+          // order by row, so that in every access below the four lanes of a quad address one row
+          float sd[4][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float4 sv = *reinterpret_cast<const float4*>(turn + (rsub + 8 * i) * kTurnPitch + csub);
-            const int owner = own_base + rsub + 8 * i;
+            const int w = i ^ qc;          // 0 -> t[0], 2 -> t[1], 1 -> t[2], 3 -> t[3]
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sd[i][e] = w == 0 ? t[0][e] : (w == 2 ? t[1][e] : (w == 1 ? t[2][e] : t[3][e]));
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int owner = own_quad + i;
             if (owner >= I.own_count) continue;
-            const int k = p + csub;
-            const float sd[4] = {sv.x, sv.y, sv.z, sv.w};
+            const int k = p + 4 * qc;
             float x[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) x[e] = k + e < r ? old[i][e] + I.coef * sd[e] : 0.f;
+            for (int e = 0; e < 4; ++e) x[e] = k + e < r ? o[i][e] + I.coef * sd[i][e] : 0.f;
             float* fp = fbase + I.own_stride * owner + I.k_stride * k;
             if (vec4) {
               if (k < r) *reinterpret_cast<float4*>(fp) = make_float4(x[0], x[1], x[2], x[3]);
@@ -317,14 +347,19 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
 #pragma unroll
             for (int e = 0; e < 4; ++e) split_bf16(x[e], h[e], l[e]);
             uint16_t* drow = dst + (int64_t)I.dst_ld * owner + k;
-            *reinterpret_cast<uint2*>(drow) = make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
-            *reinterpret_cast<uint2*>(drow + rp) = make_uint2((uint32_t)l[0] | ((uint32_t)l[1] << 16), (uint32_t)l[2] | ((uint32_t)l[3] << 16));
+            *reinterpret_cast<uint2*>(drow) =
+                make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+            *reinterpret_cast<uint2*>(drow + rp) =
+                make_uint2((uint32_t)l[0] | ((uint32_t)l[1] << 16), (uint32_t)l[2] | ((uint32_t)l[3] << 16));
           }
-          __syncwarp();
+        };
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) old[i][e] = nxt[i][e];
+        for (int pi = 0; pi < kPre; ++pi)
+          if (16 * pi < rp) piece(16 * pi, old[pi]);
+        for (int p = 16 * kPre; p < rp; p += 16) {   // ranks above 96: fetched piece by piece
+          float late[4][4];
+          fetch_old(p, late);
+          piece(p, late);
         }
       } else if (I.epi == EPI_GRAM) {
         uint16_t* dst = a.work_bf16 + I.dst_off;
