@@ -42,8 +42,9 @@ def _peaks():
 
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload
-# (profiles/ holds the captures these come from); None until captured.
-NCU_TRAFFIC_BYTES = {}
+# (profiles/ holds the captures these come from).  tc_panel: captured on the 4-layer case gpt2_1p5b@4
+# (491.4 MB per launch) and scaled by 12, since every low-rank block belongs to a layer.
+NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 12 * 491.4e6}
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
@@ -129,6 +130,24 @@ def run_reference(args) -> None:
 
 # ------------------------------------------------------------------------------------------------ GPU arm
 
+def whole_job_value(ms_local: float, steps: int, dist=None, device=None):
+    """(slowest rank's milliseconds, steps per second of the whole job).
+
+    The ranks run independent replicas of the same parameter set (the optimizer step has no exchange
+    between GPUs), so the job's throughput is all ranks' steps over the slowest rank's time.
+    `dist` is an initialised torch.distributed module or None for a single process.
+    """
+    world = 1
+    ms = float(ms_local)
+    if dist is not None:
+        import torch
+        world = dist.get_world_size()
+        t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, world * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -195,8 +214,15 @@ def kernel_algorithmic_work(kind: str, blocks, gsz: int, k_eff: int):
         fl = sum(4.0 * nb(b) * b.rank + 8.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr) / 4.0
         return "alu", fl, "flops"
     if kind == "tc_panel":
+        # g R^T and L^T g of one refit pass: 4 m n r per block (hi/lo operand doubling not counted)
         fl = sum(4.0 * nb(b) * b.rank for b in lowr)
         return "tensor", fl, "flops"
+    if kind == "tc_gram":
+        fl = sum(4.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr)
+        return "tensor", fl, "flops"
+    if kind == "tc_convert":
+        tot = sum(b.rank * (b.rows + b.cols) * (4 + 4) for b in lowr)
+        return "hbm", tot, "bytes"
     if kind in ("reduce_partial",):
         return "hbm", sum(nb(b) * gsz for b in lowr), "bytes"
     return "hbm", 0, "bytes"
@@ -223,13 +249,6 @@ def run_gpu(args) -> None:
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
 
     w = WL.get_workload(args.workload)
     blockmean = args.v_mode == "blockmean"
@@ -278,13 +297,12 @@ def run_gpu(args) -> None:
     do_steps(args.steps)
     e1.record()
     barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total, value = whole_job_value(e0.elapsed_time(e1), args.steps, dist, dev)
     clocks = sampler.stop() if sampler else None
     status = ctx.adapm_get_status()
     if status != 0:
         raise SystemExit(f"device status word {status}: a bounded wait expired; numbers are invalid")
     ms_step = ms_total / args.steps
-    value = world * args.steps / (ms_total * 1e-3)
 
     # ---- per-kernel durations (separate profiled pass; CUDA events on the launching stream) ----
     per_kind = {}
@@ -313,8 +331,8 @@ def run_gpu(args) -> None:
             params_host.copy_(params, non_blocking=True)
         e1.record()
         barrier()
-        ms_e2e = max_over_ranks(e0.elapsed_time(e1))
-        e2e = {"value": world * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": total * gsz,
+        ms_e2e, value_e2e = whole_job_value(e0.elapsed_time(e1), args.steps, dist, dev)
+        e2e = {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": total * gsz,
                "d2h_bytes_per_step": total * 4, "ms_per_step": ms_e2e / args.steps}
 
     if rank != 0:

@@ -226,3 +226,37 @@ def test_step_requires_workspace_and_aligned_pointers():
         ctx.adapm_step(params[1:], grads, state, 1)
     assert e.value.code == -2
     ctx.adapm_destroy()
+
+
+# ------------------------------------------------------------------------------------ tensor-core path
+
+def test_tensor_path_can_be_forced_and_refuses_what_it_cannot_address():
+    blocks = _pack([(256, 192, A.MOM_LOWRANK, 38, A.V_BLOCKMEAN, 0), (384, 128, A.MOM_LOWRANK, 16, A.V_ELEMENT, 0)])
+    w = WL.Workload("forced", [], "bf16", "normal", steps=5)
+    _run(w, True, 5, path=A.PATH_TENSOR, blocks=blocks)
+    # fp32 gradients cannot enter the bf16 tensor cores unchanged: the forced path is refused, AUTO falls back
+    with pytest.raises(A.AdapmError) as e:
+        A.adapm_create(blocks, A.hparams(grad_dtype=A.GRAD_F32, lowrank_path=A.PATH_TENSOR))
+    assert e.value.code == -6
+    # a row pitch that is not a multiple of 16 bytes cannot be described to the TMA unit
+    odd = _pack([(64, 130, A.MOM_LOWRANK, 4, A.V_BLOCKMEAN, 1)])
+    with pytest.raises(A.AdapmError) as e:
+        A.adapm_create(odd, A.hparams(lowrank_path=A.PATH_TENSOR))
+    assert e.value.code == -6
+
+
+def test_tensor_path_follows_moving_gradient_buffers():
+    """Tensor maps hold absolute addresses; a gradient buffer that moves between steps must be picked up."""
+    import torch
+    blocks = _pack([(256, 256, A.MOM_LOWRANK, 12, A.V_BLOCKMEAN, 1)])
+    w = WL.Workload("moving", [], "bf16", "normal", steps=4)
+    run = ParityRun(w, True, lowrank_path=A.PATH_TENSOR, custom_blocks=blocks)
+    try:
+        first = run.grads
+        for s in range(4):
+            run.grads = first if s % 2 == 0 else torch.zeros_like(first)     # a second allocation on odd steps
+            run.step()
+            run.compare()
+        assert run.ctx.adapm_get_status() == 0
+    finally:
+        run.close()
