@@ -59,13 +59,11 @@ __global__ void __launch_bounds__(256) tc_convert_kernel(const ConvertJob* __res
   for (int p = 0; p < J.rp; p += 16) {
     uint32_t h[8], l[8];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
+    for (int e = 0; e < 16; e += 2) {
       const int k = p + e;
-      const float x = k < J.r ? f[J.k_stride * k] : 0.f;
-      uint16_t a, b;
-      tc::split_bf16(x, a, b);
-      if (e & 1) { h[e >> 1] |= (uint32_t)a << 16; l[e >> 1] |= (uint32_t)b << 16; }
-      else { h[e >> 1] = a; l[e >> 1] = b; }
+      const float x0 = k < J.r ? f[J.k_stride * k] : 0.f;
+      const float x1 = k + 1 < J.r ? f[J.k_stride * (k + 1)] : 0.f;
+      tc::split_bf16x2(x0, x1, h[e >> 1], l[e >> 1]);
     }
     uint4* dh = reinterpret_cast<uint4*>(dst + p);
     uint4* dl = reinterpret_cast<uint4*>(dst + J.rp + p);

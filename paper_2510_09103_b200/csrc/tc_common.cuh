@@ -175,15 +175,21 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t smem_addr, int k16, u
 
 // ---- split bf16 --------------------------------------------------------------------------------------
 // x ~ hi + lo with both parts bf16 (round to nearest even): the pair carries about 16 significant bits.
-__device__ __forceinline__ uint16_t f32_to_bf16_rn(float x) {
-  uint32_t u = __float_as_uint(x);
-  if ((u & 0x7F800000u) == 0x7F800000u) return (uint16_t)(u >> 16);   // inf / nan: truncate
-  u += 0x7FFFu + ((u >> 16) & 1u);
-  return (uint16_t)(u >> 16);
+// Two values at a time with the packed conversion: returns {hi(x0) | hi(x1) << 16} and the same for lo.
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float x0, float x1) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(x1), "f"(x0));   // first source goes to the upper half
+  return d;
+}
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16x2_rn(x0, x1);
+  lo = pack_bf16x2_rn(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xffff0000u));
 }
 __device__ __forceinline__ void split_bf16(float x, uint16_t& hi, uint16_t& lo) {
-  hi = f32_to_bf16_rn(x);
-  lo = f32_to_bf16_rn(x - __uint_as_float((uint32_t)hi << 16));
+  uint32_t h, l;
+  split_bf16x2(x, 0.f, h, l);
+  hi = (uint16_t)(h & 0xffffu);
+  lo = (uint16_t)(l & 0xffffu);
 }
 
 }  // namespace tc

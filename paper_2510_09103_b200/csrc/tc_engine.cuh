@@ -343,14 +343,12 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
               for (int e = 0; e < 4; ++e)
                 if (k + e < r) fp[I.k_stride * e] = x[e];
             }
-            uint16_t h[4], l[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) split_bf16(x[e], h[e], l[e]);
+            uint32_t h01, l01, h23, l23;
+            split_bf16x2(x[0], x[1], h01, l01);
+            split_bf16x2(x[2], x[3], h23, l23);
             uint16_t* drow = dst + (int64_t)I.dst_ld * owner + k;
-            *reinterpret_cast<uint2*>(drow) =
-                make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
-            *reinterpret_cast<uint2*>(drow + rp) =
-                make_uint2((uint32_t)l[0] | ((uint32_t)l[1] << 16), (uint32_t)l[2] | ((uint32_t)l[3] << 16));
+            *reinterpret_cast<uint2*>(drow) = make_uint2(h01, h23);
+            *reinterpret_cast<uint2*>(drow + rp) = make_uint2(l01, l23);
           }
         };
 #pragma unroll
@@ -373,12 +371,10 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           if (q < rp) {
             uint32_t hi[8], lo[8];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float x = I.coef * ((d0[e] + d1[e]) + (d2[e] + d3[e]));
-              uint16_t h, l;
-              split_bf16(x, h, l);
-              if (e & 1) { hi[e >> 1] |= (uint32_t)h << 16; lo[e >> 1] |= (uint32_t)l << 16; }
-              else { hi[e >> 1] = h; lo[e >> 1] = l; }
+            for (int e = 0; e < 16; e += 2) {
+              const float x0 = I.coef * ((d0[e] + d1[e]) + (d2[e] + d3[e]));
+              const float x1 = I.coef * ((d0[e + 1] + d1[e + 1]) + (d2[e + 1] + d3[e + 1]));
+              split_bf16x2(x0, x1, hi[e >> 1], lo[e >> 1]);
             }
             uint4* dh = reinterpret_cast<uint4*>(dst + (int64_t)I.dst_ld * q + p);
             uint4* dl = reinterpret_cast<uint4*>(dst + (int64_t)I.dst_ld * q + rp + p);
