@@ -86,6 +86,13 @@ struct Item {
   int32_t cost;              // stages, for scheduling
 };
 
+// the fields of an Item its epilogue needs
+struct ItemEpi {
+  int32_t epi, own0, own_count, own1, col2, r, rp, dst_ld, n_dump;
+  int64_t f32_off, own_stride, k_stride, dst_off;
+  float coef;
+};
+
 struct EngineArgs {
   const Item* items;
   int32_t n_items;
@@ -234,15 +241,22 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
     const bool second = warp >= 6;                      // this warp drains the second accumulator
     int j = 0;
     for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++j) {
-      const Item& I = a.items[it];
+      // scalar fields are copied once: the stores below could alias the item table as far as the
+      // compiler can tell, and every re-read would be a round trip to global memory
+      ItemEpi I;
+      {
+        const Item& G = a.items[it];
+        I.epi = G.epi; I.own0 = G.own0; I.own_count = G.own_count; I.own1 = G.own1; I.col2 = G.col2;
+        I.r = G.r; I.rp = G.rp; I.f32_off = G.f32_off; I.own_stride = G.own_stride; I.k_stride = G.k_stride;
+        I.dst_off = G.dst_off; I.dst_ld = G.dst_ld; I.n_dump = G.n_dump; I.coef = G.coef;
+      }
       const int acc = j % a.n_acc;
       const uint32_t acc_phase = (uint32_t)(j / a.n_acc) & 1u;
       const int rp = I.rp, r = I.r;
       // EPI_FACTOR works in a "turned" layout: a thread reads its accumulator row from tensor memory,
       // then every quad of lanes transposes its 4 x 16 piece with shuffles, after which lane c of the
       // quad holds columns 4c .. 4c+3 of the quad's four rows.  Factor rows are then read and written
-      // as 64-byte runs instead of one row per lane.  The old factor values of the first kPre pieces
-      // are requested before the accumulator is waited for.
+      // as 64-byte runs instead of one row per lane.
       const bool has_work = !second || (I.epi == EPI_FACTOR && I.own1 >= 0);
       const bool factor = I.epi == EPI_FACTOR && has_work;
       const int qc = lane & 3;
@@ -266,13 +280,10 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           }
         }
       };
-      constexpr int kPre = 6;            // pieces of 16 columns whose old values are fetched up front (rp <= 96)
-      float old[kPre][4][4];
-      if (factor) {
-#pragma unroll
-        for (int pi = 0; pi < kPre; ++pi)
-          if (16 * pi < rp) fetch_old(16 * pi, old[pi]);
-      }
+      // old values travel one piece ahead in two register sets that swap roles (no copies, which
+      // would wait for the loads); the first set is requested before the accumulator is waited for
+      float oldA[4][4], oldB[4][4];
+      if (factor) fetch_old(0, oldA);
       // one lane per warp polls (fewer pollers on the barrier), then the warp agrees: the
       // tensor-memory loads below need all 32 lanes
       bool got = true;
@@ -351,13 +362,14 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             *reinterpret_cast<uint2*>(drow + rp) = make_uint2(l01, l23);
           }
         };
-#pragma unroll
-        for (int pi = 0; pi < kPre; ++pi)
-          if (16 * pi < rp) piece(16 * pi, old[pi]);
-        for (int p = 16 * kPre; p < rp; p += 16) {   // ranks above 96: fetched piece by piece
-          float late[4][4];
-          fetch_old(p, late);
-          piece(p, late);
+#pragma unroll 1
+        for (int p = 0; p < rp; p += 32) {
+          if (p + 16 < rp) fetch_old(p + 16, oldB);
+          piece(p, oldA);
+          if (p + 16 < rp) {
+            if (p + 32 < rp) fetch_old(p + 32, oldA);
+            piece(p + 16, oldB);
+          }
         }
       } else if (I.epi == EPI_GRAM) {
         uint16_t* dst = a.work_bf16 + I.dst_off;
