@@ -205,23 +205,26 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
         kr[i] = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
       }
       const int n_pieces = I.n_tiles * 4;                 // pieces of 16 columns this warp handles
-      float4 wq[4], wn[4];
+      float4 wq[4], wn[4], vq[4], vn[4];     // vq / vn: per-element v, requested with W when v is not a group scalar
       uint2 gq[4], gn[4];
       auto piece_col = [&](int gi) { return (I.tile0 + (gi >> 2)) * kApplyNT + half * 64 + (gi & 3) * 16 + csub; };
-      auto request = [&](int gi, float4* w, uint2* g) {
+      auto request = [&](int gi, float4* w, uint2* g, float4* v) {
         const int col = piece_col(gi);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const bool in = rok[i] && col + 4 <= I.cols;
           w[i] = in ? *reinterpret_cast<const float4*>(a.params + rbase[i] + col) : make_float4(0.f, 0.f, 0.f, 0.f);
           g[i] = in ? __ldg(reinterpret_cast<const uint2*>(a.grads + rbase[i] + col)) : make_uint2(0u, 0u);
+          if (!grouped)
+            v[i] = in ? *reinterpret_cast<const float4*>(a.state + I.v_off + (rbase[i] - I.off) + col)
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
         }
       };
-      request(0, wq, gq);
+      request(0, wq, gq, vq);
       for (int gi = 0; gi < n_pieces; ++gi) {
         const int jt = j + (gi >> 2), sub = gi & 3;
         const int acc = jt & 1;
-        if (gi + 1 < n_pieces) request(gi + 1, wn, gn);
+        if (gi + 1 < n_pieces) request(gi + 1, wn, gn, vn);
         if (sub == 0) {
           bool got = true;
           if (lane == 0) got = mbar_wait(&sh.tfull[acc], (uint32_t)(jt >> 1) & 1u, abort, a.status, ST_WAIT_TMEM_FULL);
@@ -256,7 +259,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
             }
           } else {
             float4* vp = reinterpret_cast<float4*>(a.state + I.v_off + (rbase[i] - I.off) + col);
-            const float4 vo = *vp;
+            const float4 vo = vq[i];
             float vv[4] = {vo.x, vo.y, vo.z, vo.w};
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
@@ -273,7 +276,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           mbar_arrive(&sh.tempty[acc]);
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { wq[i] = wn[i]; gq[i] = gn[i]; }
+        for (int i = 0; i < 4; ++i) { wq[i] = wn[i]; gq[i] = gn[i]; vq[i] = vn[i]; }
       }
       j += I.n_tiles;
     }
