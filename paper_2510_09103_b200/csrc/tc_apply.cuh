@@ -213,8 +213,8 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const bool in = rok[i] && col + 4 <= I.cols;
-          w[i] = in ? *reinterpret_cast<const float4*>(a.params + rbase[i] + col) : make_float4(0.f, 0.f, 0.f, 0.f);
-          g[i] = in ? __ldg(reinterpret_cast<const uint2*>(a.grads + rbase[i] + col)) : make_uint2(0u, 0u);
+          w[i] = in ? __ldcg(reinterpret_cast<const float4*>(a.params + rbase[i] + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          g[i] = in ? __ldcg(reinterpret_cast<const uint2*>(a.grads + rbase[i] + col)) : make_uint2(0u, 0u);
           if (!grouped)
             v[i] = in ? *reinterpret_cast<const float4*>(a.state + I.v_off + (rbase[i] - I.off) + col)
                       : make_float4(0.f, 0.f, 0.f, 0.f);
