@@ -272,11 +272,11 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           const bool row_ok = owner < I.own_count;
           const float* fp = fbase + I.own_stride * owner + I.k_stride * k;
           if (vec4) {
-            const float4 v = (row_ok && k < r) ? *reinterpret_cast<const float4*>(fp) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 v = (row_ok && k < r) ? __ldcg(reinterpret_cast<const float4*>(fp)) : make_float4(0.f, 0.f, 0.f, 0.f);
             o[i][0] = v.x; o[i][1] = v.y; o[i][2] = v.z; o[i][3] = v.w;
           } else {
 #pragma unroll
-            for (int x = 0; x < 4; ++x) o[i][x] = (row_ok && k + x < r) ? fp[I.k_stride * x] : 0.f;
+            for (int x = 0; x < 4; ++x) o[i][x] = (row_ok && k + x < r) ? __ldcg(fp + I.k_stride * x) : 0.f;
           }
         }
       };
