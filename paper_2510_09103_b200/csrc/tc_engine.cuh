@@ -44,7 +44,7 @@ constexpr int kStageK = 128;
 constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 32 KB
 constexpr int kEngineThreads = 320;
 
-enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1, EPI_DUMP = 2 };
+enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1 };
 
 struct Seg {
   int32_t map_a;             // 2-D tensor map, box 64 x 128
@@ -72,23 +72,22 @@ struct Item {
   //   dst[owner][k] = hi, dst[owner][rp + k] = lo                                      k < rp
   // EPI_GRAM: G[q][k] = coef * (D[q][k] + D[q][rp+k] + D[q][2rp+k] + D[q][3rp+k]);
   //   dst[q][k] = hi, dst[q][rp + k] = lo                                              q, k < rp
-  // EPI_DUMP: f32[q * n_dump + j] = D[q][j]                                            j < n_dump
   int32_t own0, own_count;   // first owner and number of owners of the whole matrix
   int32_t own1;              // EPI_FACTOR: first owner of the second accumulator (columns from col2), or -1
   int32_t col2;
   int32_t r, rp;
-  int64_t f32_off;           // float offset in the state buffer (EPI_DUMP: in the dump buffer)
+  int64_t f32_off;           // float offset of the factor in the state buffer
   int64_t own_stride, k_stride;
   int64_t dst_off;           // bf16 element offset of the destination array in the workspace
   int32_t dst_ld;            // its row pitch in elements
-  int32_t n_dump;
+  int32_t pad_;
   float coef;
   int32_t cost;              // stages, for scheduling
 };
 
 // the fields of an Item its epilogue needs
 struct ItemEpi {
-  int32_t epi, own0, own_count, own1, col2, r, rp, dst_ld, n_dump;
+  int32_t epi, own0, own_count, own1, col2, r, rp, dst_ld;
   int64_t f32_off, own_stride, k_stride, dst_off;
   float coef;
 };
@@ -97,7 +96,7 @@ struct EngineArgs {
   const Item* items;
   int32_t n_items;
   const CUtensorMap* maps;
-  float* f32_base;           // state buffer (or dump buffer)
+  float* f32_base;           // state buffer
   uint16_t* work_bf16;       // workspace viewed as bf16
   int32_t* status;
   int32_t stage_bytes;       // a_bytes + 16 KB * (largest number of 64-column chunks of B)
@@ -248,7 +247,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         const Item& G = a.items[it];
         I.epi = G.epi; I.own0 = G.own0; I.own_count = G.own_count; I.own1 = G.own1; I.col2 = G.col2;
         I.r = G.r; I.rp = G.rp; I.f32_off = G.f32_off; I.own_stride = G.own_stride; I.k_stride = G.k_stride;
-        I.dst_off = G.dst_off; I.dst_ld = G.dst_ld; I.n_dump = G.n_dump; I.coef = G.coef;
+        I.dst_off = G.dst_off; I.dst_ld = G.dst_ld; I.coef = G.coef;
       }
       const int acc = j % a.n_acc;
       const uint32_t acc_phase = (uint32_t)(j / a.n_acc) & 1u;
@@ -395,16 +394,6 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
           }
-        }
-      } else {   // EPI_DUMP
-        float* out = a.f32_base + I.f32_off + (int64_t)q * I.n_dump;
-        for (int p = 0; p < I.n_dump; p += 16) {
-          float d0[16];
-          tmem_ld16(t0 + (uint32_t)p, d0);
-          tmem_ld_wait();
-#pragma unroll
-          for (int e = 0; e < 16; ++e)
-            if (p + e < I.n_dump) out[p + e] = d0[e];
         }
       }
       tc_fence_before();

@@ -260,3 +260,44 @@ def test_tensor_path_follows_moving_gradient_buffers():
         assert run.ctx.adapm_get_status() == 0
     finally:
         run.close()
+
+
+def test_tensor_path_is_bitwise_reproducible():
+    import torch
+    blocks = _pack([(300, 256, A.MOM_LOWRANK, 20, A.V_BLOCKMEAN, 1), (128, 640, A.MOM_LOWRANK, 6, A.V_BLOCKMEAN, 0)])
+
+    def trajectory():
+        w = WL.Workload("repro", [], "bf16", "normal", steps=5)
+        run = ParityRun(w, True, oracle_blocks=[], lowrank_path=A.PATH_TENSOR, custom_blocks=blocks)
+        for _ in range(5):
+            run.step()
+        torch.cuda.synchronize()
+        out = run.params.clone(), run.state.clone()
+        assert run.ctx.adapm_get_status() == 0
+        run.close()
+        return out
+
+    p1, s1 = trajectory()
+    p2, s2 = trajectory()
+    assert torch.equal(p1, p2) and torch.equal(s1, s2)
+
+
+def test_tensor_path_nan_gradient_stays_in_its_block_and_does_not_hang():
+    import torch
+    blocks = _pack([(256, 128, A.MOM_LOWRANK, 8, A.V_BLOCKMEAN, 1), (128, 128, A.MOM_LOWRANK, 8, A.V_BLOCKMEAN, 1)])
+    ctx = A.adapm_create(blocks, A.hparams(lowrank_path=A.PATH_TENSOR))
+    n = blocks[1].offset + 128 * 128
+    params = torch.ones(n, device="cuda")
+    grads = torch.full((n,), 1e-3, device="cuda").bfloat16()
+    grads[7] = float("nan")                                  # inside the first block
+    state = torch.zeros(ctx.adapm_state_bytes() // 4, device="cuda")
+    work = torch.zeros(max(ctx.adapm_workspace_bytes() // 4, 64), device="cuda")
+    ctx.adapm_set_workspace(work)
+    ctx.adapm_state_init(state)
+    ctx.adapm_step(params, grads, state, 1)
+    torch.cuda.synchronize()
+    assert ctx.adapm_get_status() == 0
+    p = params.cpu().numpy()
+    assert np.isnan(p[:256 * 128]).any()
+    assert np.isfinite(p[blocks[1].offset:]).all()           # the other block never sees it
+    ctx.adapm_destroy()
