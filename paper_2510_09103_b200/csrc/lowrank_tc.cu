@@ -98,7 +98,7 @@ struct TcProgram {
     e.smem = e.n_stages * e.stage_bytes + 1024;
     return e;
   }
-  int apply_r_region = 0, apply_r_stage = 0, apply_r_stages = 1, apply_turn_off = 0;
+  int apply_r_region = 0, apply_r_stages = 3, apply_turn_off = 0;
   int n_sms = 148;
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
@@ -350,14 +350,14 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         }
       }
     }
-    // shared memory: both factor sets of the L panel, a ring of R^T tiles (one set each), the
-    // turn-around buffers of the eight epilogue warps
+    // shared memory: both factor sets of the L panel, a ring of R^T boxes, the turn-around buffers of the eight
+    // epilogue warps.  Three ring stages keep the request near 165 KB; a deeper ring was measured slower, because
+    // the shared memory it takes is L1 the epilogue's g / W loads then lack.
     const int l_region = 2 * nbc_max * tc::kBoxBytes;
     const int turn_bytes = 8 * tc::kStageFloats * 4;
-    P->apply_r_stage = nbc_max * tc::kBoxBytes;
-    P->apply_r_stages = std::max(1, std::min(4, (225 * 1024 - l_region - turn_bytes) / P->apply_r_stage));
+    P->apply_r_stages = 3;
     P->apply_r_region = l_region;
-    P->apply_turn_off = l_region + P->apply_r_stages * P->apply_r_stage;
+    P->apply_turn_off = l_region + P->apply_r_stages * tc::kBoxBytes;
     P->smem_apply = P->apply_turn_off + turn_bytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
              std::min<int64_t>((int64_t)items.size(), P->n_sms)};
@@ -449,7 +449,7 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.params = (float*)b.p[BASE_PARAMS]; a.grads = (const uint16_t*)b.p[BASE_GRADS];
       a.state = (float*)b.p[BASE_STATE]; a.status = c->d_status; a.sc = sc;
       a.use_new = sc.c1 != 0.f ? 1 : 0;
-      a.r_region_off = P->apply_r_region; a.r_stage_bytes = P->apply_r_stage; a.n_rstages = P->apply_r_stages;
+      a.r_region_off = P->apply_r_region; a.n_rstages = P->apply_r_stages;
       a.turn_off = P->apply_turn_off;
       tc::tc_apply_kernel<<<(unsigned)L.grid, tc::kApplyThreads, P->smem_apply, s>>>(a);
       break;

@@ -6,12 +6,15 @@
 //
 // An item is a 128-row panel of one block times a run of column tiles.  The split-bf16 rows of L0
 // and L of the panel stay in shared memory for the whole run; per column tile the matching rows of
-// R0^T and R^T are loaded and the products hi*hi + hi*lo + lo*hi of both factor pairs are
-// accumulated into one accumulator (the new pair with a negated A operand), so the accumulator
-// holds D = L0 R0 - L R.  Eight epilogue warps then stream g and W through registers: a thread reads
-// one accumulator row from tensor memory, the warp turns its 32 x 16 piece around through a small
+// R0^T and R^T arrive one 64-column box at a time through a ring of 16 KB stages, and every box is
+// multiplied at once with the resident L columns it pairs with (hi*hi and lo*hi for a column of the
+// hi half, hi*lo for a column of the lo half; the new pair with a negated A operand), so the
+// accumulator ends up holding D = L0 R0 - L R.  Eight epilogue warps then stream g and W through
+// registers: a thread reads one accumulator row from tensor memory, the warp turns its 32 x 16 piece around through a small
 // shared-memory buffer so that four lanes share a row, and g / W are accessed as 64-byte row
 // segments (the next piece's g and W are requested while the current one is processed).
+// The ring is kept shallow on purpose: the part of the SM's 256 KB that the CTA does not claim as
+// shared memory stays L1, and that L1 bounds how many g / W requests can be in flight.
 // The m x n matrices m_t, r_t and m^c are never stored.
 #pragma once
 
@@ -28,6 +31,7 @@ constexpr int kApplyThreads = 320;
 constexpr int kApplyNT = 128;              // columns per tile
 constexpr int kStagePitch = 20;            // floats per row of a warp's 32 x 16 turn-around buffer
 constexpr int kStageFloats = 32 * kStagePitch;
+constexpr int kApplyMaxStages = 8;         // ring depth limit
 
 struct ApplyItem {
   int64_t off;               // element offset of the block in params / grads
@@ -52,13 +56,12 @@ struct ApplyArgs {
   StepScalars sc;
   int32_t use_new;           // 0: c1 == 0, the refitted factors are not needed
   int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
-  int32_t r_stage_bytes;     // one ring stage: the R^T rows of one tile and one factor set
-  int32_t n_rstages;         // ring depth (1..4)
+  int32_t n_rstages;         // ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
   int32_t turn_off;          // byte offset of the turn-around buffers
 };
 
 struct __align__(8) ApplyShared {
-  uint64_t lfull, lempty, rfull[4], rempty[4], tfull[2], tempty[2];
+  uint64_t lfull, lempty, rfull[kApplyMaxStages], rempty[kApplyMaxStages], tfull[2], tempty[2];
   uint32_t tmem_base;
   int abort;
 };
@@ -75,7 +78,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.lfull, 1); mbar_init(&sh.lempty, 1);
-    for (int i = 0; i < 4; ++i) { mbar_init(&sh.rfull[i], 1); mbar_init(&sh.rempty[i], 1); }
+    for (int i = 0; i < kApplyMaxStages; ++i) { mbar_init(&sh.rfull[i], 1); mbar_init(&sh.rempty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 256); }
     sh.abort = 0;
     mbar_fence_init();
@@ -108,14 +111,15 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
         ++l_loads;
         for (int t = 0; t < I.n_tiles && ok; ++t) {
           const int col0 = (I.tile0 + t) * kApplyNT;
-          for (int set = 0; set < n_sets; ++set) {
-            if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
+          for (int set = 0; set < n_sets && ok; ++set) {
             const CUtensorMap* m = a.maps + (set ? I.map_r1 : I.map_r0);
-            uint8_t* dst = smem_r + (size_t)rs * a.r_stage_bytes;
-            mbar_arrive_expect_tx(&sh.rfull[rs], (uint32_t)I.nbc * kBoxBytes);
-            for (int bc = 0; bc < I.nbc; ++bc) tma_load_box(dst + (size_t)bc * kBoxBytes, m, 64 * bc, col0, &sh.rfull[rs]);
-            ++r_loads;
-            if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
+            for (int bc = 0; bc < I.nbc; ++bc) {
+              if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
+              mbar_arrive_expect_tx(&sh.rfull[rs], (uint32_t)kBoxBytes);
+              tma_load_box(smem_r + (size_t)rs * kBoxBytes, m, 64 * bc, col0, &sh.rfull[rs]);
+              ++r_loads;
+              if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
+            }
           }
         }
         item_phase ^= 1u;
@@ -152,24 +156,30 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           if (!mbar_wait(&sh.tempty[acc], acc_phase ^ 1u, abort, a.status, ST_WAIT_TMEM_EMPTY)) { ok = false; break; }
           const uint32_t d = tmem_base + (uint32_t)(acc * kApplyNT);
           uint32_t accumulate = 0;
-          for (int set = 0; set < n_sets; ++set) {
-            if (!mbar_wait(&sh.rfull[rs], rphase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
-            tc_fence_after();
+          // K step k of a [.., 2rp] operand: box k / 4 (16 KB apart), 32 bytes per step inside it
+          auto kstep = [](int k) { return (uint32_t)((k >> 2) * (kBoxBytes >> 4) + (k & 3) * 2); };
+          for (int set = 0; set < n_sets && ok; ++set) {
             const uint32_t idesc = make_idesc(kApplyNT, false, false, set == 1);
             const uint32_t la = desc_lo(l_base + (uint32_t)(set * I.nbc) * kBoxBytes, 16);
-            const uint32_t rb = desc_lo(r_base + (uint32_t)(rs * a.r_stage_bytes), 16);
-            // K step k of a [.., 2rp] operand: box k / 4 (16 KB apart), 32 bytes per step inside it
-            auto kstep = [](int k) { return (uint32_t)((k >> 2) * (kBoxBytes >> 4) + (k & 3) * 2); };
-            for (int s = 0; s < ks; ++s) {      // hi * hi
-              mma_bf16(d, desc_join(la + kstep(s), dhi), desc_join(rb + kstep(s), dhi), idesc, accumulate);
-              accumulate = 1;
+            for (int bc = 0; bc < I.nbc; ++bc) {
+              if (!mbar_wait(&sh.rfull[rs], rphase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t rb = desc_lo(r_base + (uint32_t)rs * kBoxBytes, 16);
+              for (int kk = 0; kk < 4; ++kk) {
+                const int kb = 4 * bc + kk;            // K step of [R hi | R lo] held by this box
+                if (kb >= 2 * ks) break;
+                const uint64_t b = desc_join(rb + (uint32_t)(kk * 2), dhi);
+                if (kb < ks) {                         // hi * hi, lo * hi
+                  mma_bf16(d, desc_join(la + kstep(kb), dhi), b, idesc, accumulate);
+                  mma_bf16(d, desc_join(la + kstep(ks + kb), dhi), b, idesc, 1u);
+                } else {                               // hi * lo
+                  mma_bf16(d, desc_join(la + kstep(kb - ks), dhi), b, idesc, accumulate);
+                }
+                accumulate = 1;
+              }
+              mma_commit(&sh.rempty[rs]);
+              if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
             }
-            for (int s = 0; s < ks; ++s)        // hi * lo
-              mma_bf16(d, desc_join(la + kstep(s), dhi), desc_join(rb + kstep(ks + s), dhi), idesc, 1u);
-            for (int s = 0; s < ks; ++s)        // lo * hi
-              mma_bf16(d, desc_join(la + kstep(ks + s), dhi), desc_join(rb + kstep(s), dhi), idesc, 1u);
-            mma_commit(&sh.rempty[rs]);
-            if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
           }
           if (ok) mma_commit(&sh.tfull[acc]);
         }
