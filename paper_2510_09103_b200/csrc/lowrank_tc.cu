@@ -29,8 +29,8 @@ namespace {
 
 // tensor maps of one block: g; Lc[3] and RTc[3] each as a plain matrix (A side) and as 64-column
 // chunks (N side); Gs[4] as chunks
-constexpr int kMapsPerBlock = 17;
-enum { MAP_G = 0, MAP_LC = 1, MAP_LC_N = 4, MAP_RTC = 7, MAP_RTC_N = 10, MAP_GS = 13 };
+constexpr int kMapsPerBlock = 19;
+enum { MAP_G = 0, MAP_LC = 1, MAP_LC_N = 4, MAP_RTC = 7, MAP_RTC_N = 10, MAP_GS = 13, MAP_W = 17, MAP_G32 = 18 };
 
 struct ConvertJob {
   int64_t f32_off;          // float offset of the factor in state
@@ -98,7 +98,7 @@ struct TcProgram {
     e.smem = e.n_stages * e.stage_bytes + 1024;
     return e;
   }
-  int apply_r_region = 0, apply_r_stages = 3, apply_turn_off = 0;
+  int apply_r_region = 0, apply_r_stages = 3, apply_w_region = 0, apply_bufs = 2;
   int n_sms = 148;
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
@@ -106,6 +106,7 @@ struct TcProgram {
   CUtensorMap* h_maps = nullptr;
   const void* enc_grads = nullptr;
   const void* enc_work = nullptr;
+  const void* enc_params = nullptr;
   cudaEvent_t maps_copied = nullptr;
 };
 
@@ -340,6 +341,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           a.off = b.offset; a.v_off = c->v_off[t.id]; a.rows = b.rows; a.cols = b.cols; a.r = b.rank; a.rp = t.rp;
           a.map_l0 = mb + MAP_LC; a.map_l1 = mb + MAP_LC + P->final_set;
           a.map_r0 = mb + MAP_RTC; a.map_r1 = mb + MAP_RTC + P->final_set;
+          a.map_w = mb + MAP_W; a.map_g = mb + MAP_G32;
           a.row0 = p0;
           a.tile0 = (int)((int64_t)tiles * q / runs);
           a.n_tiles = (int)((int64_t)tiles * (q + 1) / runs) - a.tile0;
@@ -350,15 +352,13 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         }
       }
     }
-    // shared memory: both factor sets of the L panel, a ring of R^T boxes, the turn-around buffers of the eight
-    // epilogue warps.  Three ring stages keep the request near 165 KB; a deeper ring was measured slower, because
-    // the shared memory it takes is L1 the epilogue's g / W loads then lack.
+    // shared memory: both factor sets of the L panel, a ring of R^T boxes, a ring of g / W quarter tiles
     const int l_region = 2 * nbc_max * tc::kBoxBytes;
-    const int turn_bytes = 8 * tc::kStageFloats * 4;
     P->apply_r_stages = 3;
     P->apply_r_region = l_region;
-    P->apply_turn_off = l_region + P->apply_r_stages * tc::kBoxBytes;
-    P->smem_apply = P->apply_turn_off + turn_bytes + 1024;
+    P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
+    P->apply_bufs = std::max(2, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / tc::kApplyBufBytes));
+    P->smem_apply = P->apply_w_region + P->apply_bufs * tc::kApplyBufBytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
              std::min<int64_t>((int64_t)items.size(), P->n_sms)};
     prog.push_back(A);
@@ -384,16 +384,18 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
 // per-step work
 // ---------------------------------------------------------------------------------------------------
 
-// Tensor maps hold absolute addresses: (re)build them when the gradient or workspace buffer moved.
+// Tensor maps hold absolute addresses: (re)build them when the parameter, gradient or workspace buffer moved.
 // The copy to the device is asynchronous on `s`; only a second move while that copy is still in
 // flight waits for it (the staging buffer is reused).
 int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
   TcProgram* P = c->tc;
   if (!P || P->blk.empty()) return ADAPM_OK;
-  if (P->enc_grads == b.p[BASE_GRADS] && P->enc_work == b.p[BASE_WORK]) return ADAPM_OK;
+  if (P->enc_grads == b.p[BASE_GRADS] && P->enc_work == b.p[BASE_WORK] && P->enc_params == b.p[BASE_PARAMS])
+    return ADAPM_OK;
   if (P->enc_grads) ADAPM_CUDA(cudaEventSynchronize(P->maps_copied));
   const char* grads = static_cast<const char*>(b.p[BASE_GRADS]);
   const char* work = static_cast<const char*>(b.p[BASE_WORK]);
+  const char* params = static_cast<const char*>(b.p[BASE_PARAMS]);
   for (size_t bi = 0; bi < P->blk.size(); ++bi) {
     const TcBlock& t = P->blk[bi];
     const adapm_block& blk = c->blocks[t.id];
@@ -401,6 +403,8 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
     const uint64_t rows = blk.rows, cols = blk.cols, rp = t.rp;
     const uint32_t nb = (uint32_t)((2 * rp + 63) / 64);
     bool ok = tc::encode_bf16_matrix(&m[MAP_G], grads + blk.offset * 2, rows, cols, cols);
+    ok = ok && tc::encode_panel32(&m[MAP_W], params + blk.offset * 4, rows, cols, true);
+    ok = ok && tc::encode_panel32(&m[MAP_G32], grads + blk.offset * 2, rows, cols, false);
     for (int q = 0; q < 3; ++q) {
       ok = ok && tc::encode_bf16_matrix(&m[MAP_LC + q], work + t.lc[q] * 2, rows, 2 * rp, 2 * rp);
       ok = ok && tc::encode_bf16_chunked(&m[MAP_LC_N + q], work + t.lc[q] * 2, rows, 2 * rp, nb, 128);
@@ -419,6 +423,7 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
   ADAPM_CUDA(cudaEventRecord(P->maps_copied, s));
   P->enc_grads = b.p[BASE_GRADS];
   P->enc_work = b.p[BASE_WORK];
+  P->enc_params = b.p[BASE_PARAMS];
   return ADAPM_OK;
 }
 
@@ -446,11 +451,10 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
     case LK_TC_APPLY: {
       tc::ApplyArgs a;
       a.items = (const tc::ApplyItem*)tab; a.n_items = (int32_t)L.n_items; a.maps = P->d_maps;
-      a.params = (float*)b.p[BASE_PARAMS]; a.grads = (const uint16_t*)b.p[BASE_GRADS];
       a.state = (float*)b.p[BASE_STATE]; a.status = c->d_status; a.sc = sc;
       a.use_new = sc.c1 != 0.f ? 1 : 0;
       a.r_region_off = P->apply_r_region; a.n_rstages = P->apply_r_stages;
-      a.turn_off = P->apply_turn_off;
+      a.w_region_off = P->apply_w_region; a.n_bufs = P->apply_bufs;
       tc::tc_apply_kernel<<<(unsigned)L.grid, tc::kApplyThreads, P->smem_apply, s>>>(a);
       break;
     }

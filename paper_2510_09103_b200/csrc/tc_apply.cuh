@@ -9,13 +9,15 @@
 // R0^T and R^T arrive one 64-column box at a time through a ring of 16 KB stages, and every box is
 // multiplied at once with the resident L columns it pairs with (hi*hi and lo*hi for a column of the
 // hi half, hi*lo for a column of the lo half; the new pair with a negated A operand), so the
-// accumulator ends up holding D = L0 R0 - L R.  Eight epilogue warps then stream g and W through
-// registers: a thread reads one accumulator row from tensor memory, the warp turns its 32 x 16 piece around through a small
-// shared-memory buffer so that four lanes share a row, and g / W are accessed as 64-byte row
-// segments (the next piece's g and W are requested while the current one is processed).
-// The ring is kept shallow on purpose: the part of the SM's 256 KB that the CTA does not claim as
-// shared memory stays L1, and that L1 bounds how many g / W requests can be in flight.
-// The m x n matrices m_t, r_t and m^c are never stored.
+// accumulator ends up holding D = L0 R0 - L R.
+//
+// g and W never pass through registers on their way in or out: a mover thread brings them in
+// quarter tiles (128 rows x 32 columns: 16 KB of W, 8 KB of g) by TMA into a small ring of
+// shared-memory buffers, several quarters ahead of their use, and writes the updated W back from
+// the same buffer by TMA.  Each of the 256 epilogue threads owns one row of the panel: it reads its
+// accumulator row from tensor memory, its 16 columns of g and W from the (swizzled) buffer, and
+// puts the new W back in place.  Only a per-element v, where a block has one, is read and written
+// directly.  The m x n matrices m_t, r_t and m^c are never stored.
 #pragma once
 
 #include <cuda.h>
@@ -27,17 +29,21 @@
 namespace adapm {
 namespace tc {
 
-constexpr int kApplyThreads = 320;
+constexpr int kApplyThreads = 352;         // producer warp, MMA warp, eight epilogue warps, mover warp
 constexpr int kApplyNT = 128;              // columns per tile
-constexpr int kStagePitch = 20;            // floats per row of a warp's 32 x 16 turn-around buffer
-constexpr int kStageFloats = 32 * kStagePitch;
-constexpr int kApplyMaxStages = 8;         // ring depth limit
+constexpr int kApplyQC = 32;               // columns per quarter tile
+constexpr int kApplyMaxStages = 8;         // R ring depth limit
+constexpr int kApplyMaxBufs = 4;           // g / W ring depth limit
+constexpr int kWBoxBytes = 128 * kApplyQC * 4;   // a quarter tile of W: 128 rows of 128 bytes
+constexpr int kGBoxBytes = 128 * kApplyQC * 2;   // and of g: 128 rows of 64 bytes
+constexpr int kApplyBufBytes = kWBoxBytes + kGBoxBytes;
 
 struct ApplyItem {
   int64_t off;               // element offset of the block in params / grads
   int64_t v_off;             // float offset of v in state
   int32_t rows, cols, r, rp;
   int32_t map_l0, map_l1, map_r0, map_r1;   // split factors: [rows, 2rp] and [cols, 2rp], boxes of 64 x 128
+  int32_t map_w, map_g;      // params and grads of the block, boxes of 32 x 128
   int32_t row0;              // first row of the panel
   int32_t tile0, n_tiles;    // column tiles [tile0, tile0 + n_tiles) of 128 columns
   int32_t nbc;               // 64-wide boxes across the 2rp split columns
@@ -49,19 +55,20 @@ struct ApplyArgs {
   const ApplyItem* items;
   int32_t n_items;
   const CUtensorMap* maps;
-  float* params;
-  const uint16_t* grads;
   float* state;
   int32_t* status;
   StepScalars sc;
   int32_t use_new;           // 0: c1 == 0, the refitted factors are not needed
   int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
-  int32_t n_rstages;         // ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
-  int32_t turn_off;          // byte offset of the turn-around buffers
+  int32_t n_rstages;         // R ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
+  int32_t w_region_off;      // byte offset of the g / W ring
+  int32_t n_bufs;            // g / W ring depth (2..kApplyMaxBufs); a buffer is kApplyBufBytes
 };
 
 struct __align__(8) ApplyShared {
   uint64_t lfull, lempty, rfull[kApplyMaxStages], rempty[kApplyMaxStages], tfull[2], tempty[2];
+  uint64_t wfull[kApplyMaxBufs];   // a quarter's g and W have landed
+  uint64_t wdone[kApplyMaxBufs];   // all 256 epilogue threads have put their new W back
   uint32_t tmem_base;
   int abort;
 };
@@ -72,6 +79,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dyn_smem) + 1023) & ~(uintptr_t)1023);
   uint8_t* smem_l = smem;
   uint8_t* smem_r = smem + a.r_region_off;
+  uint8_t* smem_w = smem + a.w_region_off;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort = &sh.abort;
   const int n_sets = a.use_new ? 2 : 1;
@@ -80,6 +88,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
     mbar_init(&sh.lfull, 1); mbar_init(&sh.lempty, 1);
     for (int i = 0; i < kApplyMaxStages; ++i) { mbar_init(&sh.rfull[i], 1); mbar_init(&sh.rempty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 256); }
+    for (int i = 0; i < kApplyMaxBufs; ++i) { mbar_init(&sh.wfull[i], 1); mbar_init(&sh.wdone[i], 256); }
     sh.abort = 0;
     mbar_fence_init();
   }
@@ -187,55 +196,102 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
         item_phase ^= 1u;
       }
     }
+  } else if (warp == 10) {
+    // ------------------------------------------------------------------ g / W mover
+    if (lane == 0) {
+      // load cursor: runs n_bufs - 1 quarters ahead of the quarter being stored
+      int ld_it = blockIdx.x, ld_q = 0, ld_nq = 0, n_loaded = 0;
+      ApplyItem LI;
+      if (ld_it < a.n_items) { LI = a.items[ld_it]; ld_nq = 4 * LI.n_tiles; }
+      auto load_next = [&]() {
+        const int b = n_loaded % a.n_bufs;
+        uint8_t* buf = smem_w + (size_t)b * kApplyBufBytes;
+        const int col = (LI.tile0 + (ld_q >> 2)) * kApplyNT + (ld_q & 3) * kApplyQC;
+        mbar_arrive_expect_tx(&sh.wfull[b], (uint32_t)kApplyBufBytes);
+        tma_load_box(buf, a.maps + LI.map_w, col, LI.row0, &sh.wfull[b]);
+        tma_load_box(buf + kWBoxBytes, a.maps + LI.map_g, col, LI.row0, &sh.wfull[b]);
+        ++n_loaded;
+        if (++ld_q == ld_nq) {
+          ld_it += gridDim.x; ld_q = 0; ld_nq = 0;
+          if (ld_it < a.n_items) { LI = a.items[ld_it]; ld_nq = 4 * LI.n_tiles; }
+        }
+      };
+      for (int i = 0; i + 1 < a.n_bufs && ld_it < a.n_items; ++i) load_next();
+      int k = 0;   // running quarter count of this CTA
+      bool ok = true;
+      for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
+        const ApplyItem I = a.items[it];
+        for (int q = 0; q < 4 * I.n_tiles; ++q, ++k) {
+          const int b = k % a.n_bufs;
+          if (!mbar_wait(&sh.wdone[b], (uint32_t)(k / a.n_bufs) & 1u, abort, a.status, ST_WAIT_DRAIN)) { ok = false; break; }
+          const int col = (I.tile0 + (q >> 2)) * kApplyNT + (q & 3) * kApplyQC;
+          // (a quarter that lies past the last column is not stored; its group is committed empty, so
+          // that the count below still means "the store before this one")
+          if (col < I.cols) tma_store_box(a.maps + I.map_w, col, I.row0, smem_w + (size_t)b * kApplyBufBytes);
+          bulk_commit_group();
+          if (ld_it < a.n_items) {
+            // the next load goes into the buffer stored one quarter ago: wait until that store has
+            // read it (every group but the one just committed)
+            bulk_wait_group_read<1>();
+            load_next();
+          }
+        }
+      }
+      bulk_wait_group<0>();
+      if (!ok) {   // let the loads already issued land before the CTA exits
+        for (int kk = k; kk < n_loaded; ++kk) {
+          const uint32_t ph = (uint32_t)(kk / a.n_bufs) & 1u;
+          for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&sh.wfull[kk % a.n_bufs], ph); ++spin)
+            __nanosleep(64);
+        }
+      }
+    }
   } else {
     // ------------------------------------------------------------------ epilogue
     const int e = warp - 2;
     const int wq4 = warp & 3;                             // which 32 accumulator rows this warp may read
-    const int half = e >> 2;                              // which 64 columns of the tile
+    const int half = e >> 2;                              // which 16 columns of a quarter
     const uint32_t lane_addr = (uint32_t)(32 * wq4) << 16;
-    float* turn = reinterpret_cast<float*>(smem + a.turn_off) + e * kStageFloats;
+    const int rloc = 32 * wq4 + lane;                     // this thread's row of the panel
     const StepScalars sc = a.sc;
-    const int rsub = lane >> 2;                           // after the turn: row rsub + 8 i, i = 0..3
-    const int csub = 4 * (lane & 3);                      // and four columns starting here
-    int j = 0;
+    // byte offsets of this thread's 16-byte chunks inside a buffer: the 128-byte swizzle turns chunk c of
+    // row r into chunk c ^ (r % 8), the 64-byte swizzle chunk c of a 64-byte row into c ^ ((r / 2) % 4)
+    uint32_t w_at[4], g_at[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w_at[i] = (uint32_t)(rloc * 128 + (((4 * half + i) ^ (rloc & 7)) << 4));
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      g_at[i] = (uint32_t)(kWBoxBytes + rloc * 64 + (((2 * half + i) ^ ((rloc >> 1) & 3)) << 4));
+    int j = 0, k = 0;   // running tile and quarter counts of this CTA
     bool ok = true;
     for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
       const ApplyItem I = a.items[it];
       const bool grouped = I.v_mode == ADAPM_V_BLOCKMEAN;
       const float lr_s = sc.lr * I.lr_scale;
-      int64_t rbase[4];
-      bool rok[4];
-      float kr[4];   // one denominator per row when v is a group scalar: m^c / (sqrt(v) + eps) becomes a product
+      const int row = I.row0 + rloc;
+      const bool rok = row < I.rows;
+      // one denominator per row when v is a group scalar: m^c / (sqrt(v) + eps) becomes a product
+      const float v_row = (rok && grouped) ? a.state[I.v_off + row / I.v_group_rows] : 0.f;
+      const float kr = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
+      float* vrow = a.state + I.v_off + (int64_t)row * I.cols;   // per-element v of this row (not grouped)
+      const int n_q = 4 * I.n_tiles;
+      auto v_col = [&](int q) { return (I.tile0 + (q >> 2)) * kApplyNT + (q & 3) * kApplyQC + 16 * half; };
+      auto v_fetch = [&](int q, float4* v) {
+        const int col = v_col(q);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int row = I.row0 + 32 * wq4 + rsub + 8 * i;
-        rok[i] = row < I.rows;
-        rbase[i] = I.off + (int64_t)row * I.cols;
-        const float v_row = (rok[i] && grouped) ? a.state[I.v_off + row / I.v_group_rows] : 0.f;
-        kr[i] = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
-      }
-      const int n_pieces = I.n_tiles * 4;                 // pieces of 16 columns this warp handles
-      float4 wq[4], wn[4], vq[4], vn[4];     // vq / vn: per-element v, requested with W when v is not a group scalar
-      uint2 gq[4], gn[4];
-      auto piece_col = [&](int gi) { return (I.tile0 + (gi >> 2)) * kApplyNT + half * 64 + (gi & 3) * 16 + csub; };
-      auto request = [&](int gi, float4* w, uint2* g, float4* v) {
-        const int col = piece_col(gi);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const bool in = rok[i] && col + 4 <= I.cols;
-          w[i] = in ? __ldcg(reinterpret_cast<const float4*>(a.params + rbase[i] + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          g[i] = in ? __ldcg(reinterpret_cast<const uint2*>(a.grads + rbase[i] + col)) : make_uint2(0u, 0u);
-          if (!grouped)
-            v[i] = in ? *reinterpret_cast<const float4*>(a.state + I.v_off + (rbase[i] - I.off) + col)
-                      : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+        for (int i = 0; i < 4; ++i)
+          v[i] = (rok && col + 4 * i + 4 <= I.cols) ? __ldcg(reinterpret_cast<const float4*>(vrow + col) + i)
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
       };
-      request(0, wq, gq, vq);
-      for (int gi = 0; gi < n_pieces; ++gi) {
-        const int jt = j + (gi >> 2), sub = gi & 3;
+      float4 vq[4], vn[4];
+      if (!grouped) v_fetch(0, vq);
+      for (int q = 0; q < n_q; ++q, ++k) {
+        const int jt = j + (q >> 2), sub = q & 3;
         const int acc = jt & 1;
-        if (gi + 1 < n_pieces) request(gi + 1, wn, gn, vn);
+        const int b = k % a.n_bufs;
+        if (!grouped && q + 1 < n_q) v_fetch(q + 1, vn);
         if (sub == 0) {
+          // one lane per warp polls, then the warp agrees: the tensor-memory loads need all 32 lanes
           bool got = true;
           if (lane == 0) got = mbar_wait(&sh.tfull[acc], (uint32_t)(jt >> 1) & 1u, abort, a.status, ST_WAIT_TMEM_FULL);
           got = __shfl_sync(0xffffffffu, got, 0);
@@ -243,50 +299,59 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           tc_fence_after();
         }
         float d[16];
-        tmem_ld16(tmem_base + lane_addr + (uint32_t)(acc * kApplyNT + half * 64 + sub * 16), d);
+        tmem_ld16(tmem_base + lane_addr + (uint32_t)(acc * kApplyNT + sub * kApplyQC + 16 * half), d);
+        if (!mbar_wait(&sh.wfull[b], (uint32_t)(k / a.n_bufs) & 1u, abort, a.status, ST_WAIT_FULL)) ok = false;
+        ok = __all_sync(0xffffffffu, ok);
         tmem_ld_wait();
-        float4* mine = reinterpret_cast<float4*>(turn + lane * kStagePitch);
-        mine[0] = make_float4(d[0], d[1], d[2], d[3]);
-        mine[1] = make_float4(d[4], d[5], d[6], d[7]);
-        mine[2] = make_float4(d[8], d[9], d[10], d[11]);
-        mine[3] = make_float4(d[12], d[13], d[14], d[15]);
-        __syncwarp();
-        const int col = piece_col(gi);
+        if (!ok) break;
+        uint8_t* buf = smem_w + (size_t)b * kApplyBufBytes;
+        float gf[16];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const uint4 gg = *reinterpret_cast<const uint4*>(buf + g_at[i]);
+          const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w};
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            gf[8 * i + 2 * x] = __uint_as_float(gw[x] << 16);
+            gf[8 * i + 2 * x + 1] = __uint_as_float(gw[x] & 0xffff0000u);
+          }
+        }
+        const int col = v_col(q);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float4 dv = *reinterpret_cast<const float4*>(turn + (rsub + 8 * i) * kStagePitch + csub);
-          if (!(rok[i] && col + 4 <= I.cols)) continue;
-          const float dd[4] = {dv.x, dv.y, dv.z, dv.w};
-          const float gf[4] = {__uint_as_float(gq[i].x << 16), __uint_as_float(gq[i].x & 0xffff0000u),
-                               __uint_as_float(gq[i].y << 16), __uint_as_float(gq[i].y & 0xffff0000u)};
-          float w[4] = {wq[i].x, wq[i].y, wq[i].z, wq[i].w};
+          float4* wp = reinterpret_cast<float4*>(buf + w_at[i]);
+          const float4 wo = *wp;
+          float w[4] = {wo.x, wo.y, wo.z, wo.w};
           if (grouped) {
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
-              float ratio = (sc.cg * gf[x] + sc.c0 * dd[x]) * kr[i];
+              float ratio = (sc.cg * gf[4 * i + x] + sc.c0 * d[4 * i + x]) * kr;
               ratio = ratio > sc.clip ? sc.clip : (ratio < -sc.clip ? -sc.clip : ratio);
               w[x] = w[x] - lr_s * (ratio + I.wd * w[x]);
             }
           } else {
-            float4* vp = reinterpret_cast<float4*>(a.state + I.v_off + (rbase[i] - I.off) + col);
-            const float4 vo = vq[i];
-            float vv[4] = {vo.x, vo.y, vo.z, vo.w};
+            float vv[4] = {vq[i].x, vq[i].y, vq[i].z, vq[i].w};
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
-              vv[x] = sc.beta2 * vv[x] + (1.f - sc.beta2) * (gf[x] * gf[x]);
-              w[x] = adapm_param_update(w[x], sc.cg * gf[x] + sc.c0 * dd[x], vv[x], sc, lr_s, I.wd);
+              const float g1 = gf[4 * i + x];
+              vv[x] = sc.beta2 * vv[x] + (1.f - sc.beta2) * (g1 * g1);
+              w[x] = adapm_param_update(w[x], sc.cg * g1 + sc.c0 * d[4 * i + x], vv[x], sc, lr_s, I.wd);
             }
-            *vp = make_float4(vv[0], vv[1], vv[2], vv[3]);
+            if (rok && col + 4 * i + 4 <= I.cols)
+              *(reinterpret_cast<float4*>(vrow + col) + i) = make_float4(vv[0], vv[1], vv[2], vv[3]);
           }
-          *reinterpret_cast<float4*>(a.params + rbase[i] + col) = make_float4(w[0], w[1], w[2], w[3]);
+          *wp = make_float4(w[0], w[1], w[2], w[3]);
         }
-        __syncwarp();
+        fence_async_smem();
+        mbar_arrive(&sh.wdone[b]);
         if (sub == 3) {
           tc_fence_before();
           mbar_arrive(&sh.tempty[acc]);
         }
+        if (!grouped) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) { wq[i] = wn[i]; gq[i] = gn[i]; vq[i] = vn[i]; }
+          for (int i = 0; i < 4; ++i) vq[i] = vn[i];
+        }
       }
       j += I.n_tiles;
     }

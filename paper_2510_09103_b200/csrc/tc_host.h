@@ -58,5 +58,22 @@ inline bool encode_bf16_chunked(CUtensorMap* out, const void* base, uint64_t row
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of a row-major matrix [rows, cols] of 2- or 4-byte elements (row pitch = cols), moved in
+// boxes of 32 columns x 128 rows: 128-byte swizzle for fp32 (128-byte box rows), 64-byte swizzle
+// for bf16 (64-byte box rows).  Loads read zero out of range, stores skip what is out of range.
+// Requires: base 16-byte aligned, cols * element size a multiple of 16 bytes.
+inline bool encode_panel32(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, bool is_f32) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * (is_f32 ? 4u : 2u)};
+  const cuuint32_t box[2] = {32, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(out, is_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            is_f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tc
 }  // namespace adapm
