@@ -98,7 +98,7 @@ struct TcProgram {
     e.smem = e.n_stages * e.stage_bytes + 1024;
     return e;
   }
-  int apply_r_region = 0, apply_r_stages = 3, apply_w_region = 0, apply_bufs = 2;
+  int apply_r_region = 0, apply_r_stages = 2, apply_w_region = 0, apply_bufs = 2;
   int n_sms = 148;
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
@@ -354,10 +354,10 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     }
     // shared memory: both factor sets of the L panel, a ring of R^T boxes, a ring of g / W quarter tiles
     const int l_region = 2 * nbc_max * tc::kBoxBytes;
-    P->apply_r_stages = 3;
+    P->apply_r_stages = 2;   // (a deeper R ring measured no faster; the g / W ring is what pays)
     P->apply_r_region = l_region;
     P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
-    P->apply_bufs = std::max(2, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / tc::kApplyBufBytes));
+    P->apply_bufs = std::max(1, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / tc::kApplyBufBytes));
     P->smem_apply = P->apply_w_region + P->apply_bufs * tc::kApplyBufBytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
              std::min<int64_t>((int64_t)items.size(), P->n_sms)};

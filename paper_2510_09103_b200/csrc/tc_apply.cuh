@@ -33,7 +33,7 @@ constexpr int kApplyThreads = 352;         // producer warp, MMA warp, eight epi
 constexpr int kApplyNT = 128;              // columns per tile
 constexpr int kApplyQC = 32;               // columns per quarter tile
 constexpr int kApplyMaxStages = 8;         // R ring depth limit
-constexpr int kApplyMaxBufs = 4;           // g / W ring depth limit
+constexpr int kApplyMaxBufs = 6;           // g / W ring depth limit
 constexpr int kWBoxBytes = 128 * kApplyQC * 4;   // a quarter tile of W: 128 rows of 128 bytes
 constexpr int kGBoxBytes = 128 * kApplyQC * 2;   // and of g: 128 rows of 64 bytes
 constexpr int kApplyBufBytes = kWBoxBytes + kGBoxBytes;
@@ -62,13 +62,13 @@ struct ApplyArgs {
   int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
   int32_t n_rstages;         // R ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
   int32_t w_region_off;      // byte offset of the g / W ring
-  int32_t n_bufs;            // g / W ring depth (2..kApplyMaxBufs); a buffer is kApplyBufBytes
+  int32_t n_bufs;            // g / W ring depth (1..kApplyMaxBufs); a buffer is kApplyBufBytes
 };
 
 struct __align__(8) ApplyShared {
   uint64_t lfull, lempty, rfull[kApplyMaxStages], rempty[kApplyMaxStages], tfull[2], tempty[2];
   uint64_t wfull[kApplyMaxBufs];   // a quarter's g and W have landed
-  uint64_t wdone[kApplyMaxBufs];   // all 256 epilogue threads have put their new W back
+  uint64_t wdone[kApplyMaxBufs];   // all eight epilogue warps have put their new W back
   uint32_t tmem_base;
   int abort;
 };
@@ -87,8 +87,8 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
   if (threadIdx.x == 0) {
     mbar_init(&sh.lfull, 1); mbar_init(&sh.lempty, 1);
     for (int i = 0; i < kApplyMaxStages; ++i) { mbar_init(&sh.rfull[i], 1); mbar_init(&sh.rempty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 256); }
-    for (int i = 0; i < kApplyMaxBufs; ++i) { mbar_init(&sh.wfull[i], 1); mbar_init(&sh.wdone[i], 256); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 8); }
+    for (int i = 0; i < kApplyMaxBufs; ++i) { mbar_init(&sh.wfull[i], 1); mbar_init(&sh.wdone[i], 8); }
     sh.abort = 0;
     mbar_fence_init();
   }
@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
   } else if (warp == 10) {
     // ------------------------------------------------------------------ g / W mover
     if (lane == 0) {
-      // load cursor: runs n_bufs - 1 quarters ahead of the quarter being stored
+      // load cursor: runs n_bufs quarters ahead of the quarter being stored
       int ld_it = blockIdx.x, ld_q = 0, ld_nq = 0, n_loaded = 0;
       ApplyItem LI;
       if (ld_it < a.n_items) { LI = a.items[ld_it]; ld_nq = 4 * LI.n_tiles; }
@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           if (ld_it < a.n_items) { LI = a.items[ld_it]; ld_nq = 4 * LI.n_tiles; }
         }
       };
-      for (int i = 0; i + 1 < a.n_bufs && ld_it < a.n_items; ++i) load_next();
+      for (int i = 0; i < a.n_bufs && ld_it < a.n_items; ++i) load_next();
       int k = 0;   // running quarter count of this CTA
       bool ok = true;
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
@@ -225,14 +225,12 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           const int b = k % a.n_bufs;
           if (!mbar_wait(&sh.wdone[b], (uint32_t)(k / a.n_bufs) & 1u, abort, a.status, ST_WAIT_DRAIN)) { ok = false; break; }
           const int col = (I.tile0 + (q >> 2)) * kApplyNT + (q & 3) * kApplyQC;
-          // (a quarter that lies past the last column is not stored; its group is committed empty, so
-          // that the count below still means "the store before this one")
+          // (a quarter that lies past the last column is not stored)
           if (col < I.cols) tma_store_box(a.maps + I.map_w, col, I.row0, smem_w + (size_t)b * kApplyBufBytes);
           bulk_commit_group();
           if (ld_it < a.n_items) {
-            // the next load goes into the buffer stored one quarter ago: wait until that store has
-            // read it (every group but the one just committed)
-            bulk_wait_group_read<1>();
+            // the next load goes into this same buffer, as soon as the store has read it
+            bulk_wait_group_read<0>();
             load_next();
           }
         }
@@ -342,11 +340,13 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           }
           *wp = make_float4(w[0], w[1], w[2], w[3]);
         }
+        // one arrival per warp: every lane orders its own writes (and tensor-memory reads), the warp meets
         fence_async_smem();
-        mbar_arrive(&sh.wdone[b]);
-        if (sub == 3) {
-          tc_fence_before();
-          mbar_arrive(&sh.tempty[acc]);
+        if (sub == 3) tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&sh.wdone[b]);
+          if (sub == 3) mbar_arrive(&sh.tempty[acc]);
         }
         if (!grouped) {
 #pragma unroll
