@@ -228,10 +228,13 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           // (a quarter that lies past the last column is not stored)
           if (col < I.cols) tma_store_box(a.maps + I.map_w, col, I.row0, smem_w + (size_t)b * kApplyBufBytes);
           bulk_commit_group();
-          if (ld_it < a.n_items) {
-            // the next load goes into this same buffer, as soon as the store has read it
+          if ((k & 1) && ld_it < a.n_items) {
+            // two quarters at a time: their rows are neighbours in memory, and requests that reach DRAM
+            // together share its open pages.  They go into this buffer and the one stored before it,
+            // once both stores have read them.
             bulk_wait_group_read<0>();
             load_next();
+            if (ld_it < a.n_items) load_next();
           }
         }
       }
