@@ -28,20 +28,22 @@ void set_error_text(const char* text);   // ctx.cu
 namespace {
 
 // tensor maps of one block: g; Lc[3] and RTc[3] each as a plain matrix (A side) and as 64-column
-// chunks (N side); Gs[4] as chunks
-constexpr int kMapsPerBlock = 19;
-enum { MAP_G = 0, MAP_LC = 1, MAP_LC_N = 4, MAP_RTC = 7, MAP_RTC_N = 10, MAP_GS = 13, MAP_W = 17, MAP_G32 = 18 };
+// chunks (N side); Gs[4] as chunks; W and g in quarter-tile boxes; the previous and the final set of
+// Lc and of RTc side by side as one matrix (the apply kernel's operands)
+constexpr int kMapsPerBlock = 21;
+enum { MAP_G = 0, MAP_LC = 1, MAP_LC_N = 4, MAP_RTC = 7, MAP_RTC_N = 10, MAP_GS = 13, MAP_W = 17, MAP_G32 = 18,
+       MAP_LCAT = 19, MAP_RCAT = 20 };
 
 struct ConvertJob {
   int64_t f32_off;          // float offset of the factor in state
   int64_t own_stride, k_stride;
   int64_t dst_off;          // bf16 element offset in the workspace
   int32_t owners, r, rp;
-  int32_t pad_;
+  int32_t dst_ld;           // row pitch of the destination, in elements
   int64_t first_owner;      // prefix sum of owners
 };
 
-// fp32 factor -> [owners, 2rp] split bf16 (hi columns, then lo columns; columns >= r are zero)
+// fp32 factor -> [owners, 2rp] split bf16 with row pitch dst_ld (hi columns, then lo columns; columns >= r are zero)
 __global__ void __launch_bounds__(256) tc_convert_kernel(const ConvertJob* __restrict__ jobs, int n_jobs,
                                                          int64_t total_owners, const float* __restrict__ state,
                                                          uint16_t* __restrict__ work) {
@@ -55,7 +57,7 @@ __global__ void __launch_bounds__(256) tc_convert_kernel(const ConvertJob* __res
   const ConvertJob J = jobs[lo];
   const int64_t owner = gid - J.first_owner;
   const float* f = state + J.f32_off + J.own_stride * owner;
-  uint16_t* dst = work + J.dst_off + (int64_t)(2 * J.rp) * owner;
+  uint16_t* dst = work + J.dst_off + (int64_t)J.dst_ld * owner;
   for (int p = 0; p < J.rp; p += 16) {
     uint32_t h[8], l[8];
 #pragma unroll
@@ -81,6 +83,7 @@ struct TcBlock {
   int64_t id;                      // index into ctx->blocks
   int32_t rp;
   int64_t lc[3], rtc[3], gs[4];    // bf16 element offsets in the workspace
+  int32_t ld[3];                   // row pitch of set s of lc / rtc, in elements
 };
 
 struct TcProgram {
@@ -98,7 +101,7 @@ struct TcProgram {
     e.smem = e.n_stages * e.stage_bytes + 1024;
     return e;
   }
-  int apply_r_region = 0, apply_r_stages = 2, apply_w_region = 0, apply_bufs = 2;
+  int apply_r_region = 0, apply_r_stages = 3, apply_w_region = 0, apply_bufs = 2;
   int n_sms = 148;
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
@@ -193,6 +196,10 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     work_cursor += round_up((bf16_elems + 128 + 1) / 2, kStateAlign);   // +256 B: see encode_bf16_chunked
     return off;
   };
+  // the refit passes alternate between sets 1 and 2, starting from 0.  Without any pass the "final" factors are
+  // the previous ones: they are then converted a second time, into set 1, so that the apply kernel's operand
+  // layout does not change.
+  P->final_set = etas.empty() ? 1 : (etas.size() % 2 ? 1 : 2);
   int rp_max = 16;
   for (int64_t id : tc_ids) {
     const adapm_block& b = c->blocks[id];
@@ -200,8 +207,13 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     t.id = id;
     t.rp = round16(b.rank);
     rp_max = std::max(rp_max, t.rp);
-    for (int s = 0; s < 3; ++s) t.lc[s] = take((int64_t)b.rows * 2 * t.rp);
-    for (int s = 0; s < 3; ++s) t.rtc[s] = take((int64_t)b.cols * 2 * t.rp);
+    // the previous set (0) and the set the last refit pass writes share one array with row pitch 4rp, side by
+    // side, so that the apply kernel reads both as one 4rp-wide operand; the third set has an array of its own
+    const int64_t lcat = take((int64_t)b.rows * 4 * t.rp), rcat = take((int64_t)b.cols * 4 * t.rp);
+    const int other = 3 - P->final_set;
+    t.lc[0] = lcat; t.lc[P->final_set] = lcat + 2 * t.rp; t.lc[other] = take((int64_t)b.rows * 2 * t.rp);
+    t.rtc[0] = rcat; t.rtc[P->final_set] = rcat + 2 * t.rp; t.rtc[other] = take((int64_t)b.cols * 2 * t.rp);
+    for (int s = 0; s < 3; ++s) t.ld[s] = (s == other ? 2 : 4) * t.rp;
     for (int w = 0; w < 4; ++w) t.gs[w] = take((int64_t)2 * t.rp * t.rp);
     P->blk.push_back(t);
   }
@@ -228,10 +240,13 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       ConvertJob j;
       std::memset(&j, 0, sizeof(j));
       j.r = b.rank; j.rp = t.rp;
-      j.f32_off = c->l_off[t.id]; j.own_stride = b.rank; j.k_stride = 1; j.owners = b.rows; j.dst_off = t.lc[0];
-      j.first_owner = owners; owners += j.owners; jobs.push_back(j);
-      j.f32_off = c->r_off[t.id]; j.own_stride = 1; j.k_stride = b.cols; j.owners = b.cols; j.dst_off = t.rtc[0];
-      j.first_owner = owners; owners += j.owners; jobs.push_back(j);
+      j.dst_ld = 4 * t.rp;   // sets 0 and (without refit passes) 1 = the final set: the shared array
+      for (int set = 0; set < (etas.empty() ? 2 : 1); ++set) {
+        j.f32_off = c->l_off[t.id]; j.own_stride = b.rank; j.k_stride = 1; j.owners = b.rows; j.dst_off = t.lc[set];
+        j.first_owner = owners; owners += j.owners; jobs.push_back(j);
+        j.f32_off = c->r_off[t.id]; j.own_stride = 1; j.k_stride = b.cols; j.owners = b.cols; j.dst_off = t.rtc[set];
+        j.first_owner = owners; owners += j.owners; jobs.push_back(j);
+      }
     }
     P->n_convert_owners = owners;
     Launch L{LK_TC_CONVERT, append_items(c->h_tables, jobs), (int64_t)jobs.size(), (owners + 255) / 256};
@@ -300,7 +315,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         it.own0 = p0; it.own_count = is_L ? m : n;
         it.f32_off = is_L ? c->l_off[t.id] : c->r_off[t.id];
         it.own_stride = is_L ? r : 1; it.k_stride = is_L ? 1 : n;
-        it.dst_off = is_L ? t.lc[dst] : t.rtc[dst]; it.dst_ld = 2 * rp;
+        it.dst_off = is_L ? t.lc[dst] : t.rtc[dst]; it.dst_ld = t.ld[dst];
         panels.push_back(it);
       };
       const int step = pair_panels ? 256 : 128;
@@ -320,7 +335,6 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     prog.push_back(Q);
     src = dst;
   }
-  P->final_set = src;
 
   // ---- apply ---------------------------------------------------------------------------------------------------
   {
@@ -330,8 +344,8 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       const TcBlock& t = P->blk[bi];
       const adapm_block& b = c->blocks[t.id];
       const int mb = (int)bi * kMapsPerBlock;
-      const int nbc = (2 * t.rp + 63) / 64;
-      nbc_max = std::max(nbc_max, nbc);
+      const int nbc1 = (2 * t.rp + 63) / 64, nbc2 = (4 * t.rp + 63) / 64;
+      nbc_max = std::max(nbc_max, nbc2);
       const int tiles = (b.cols + tc::kApplyNT - 1) / tc::kApplyNT;
       const int runs = (tiles + 15) / 16;
       for (int p0 = 0; p0 < b.rows; p0 += 128) {
@@ -339,25 +353,26 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           tc::ApplyItem a;
           std::memset(&a, 0, sizeof(a));
           a.off = b.offset; a.v_off = c->v_off[t.id]; a.rows = b.rows; a.cols = b.cols; a.r = b.rank; a.rp = t.rp;
-          a.map_l0 = mb + MAP_LC; a.map_l1 = mb + MAP_LC + P->final_set;
-          a.map_r0 = mb + MAP_RTC; a.map_r1 = mb + MAP_RTC + P->final_set;
+          a.map_l = mb + MAP_LCAT; a.map_r = mb + MAP_RCAT;
           a.map_w = mb + MAP_W; a.map_g = mb + MAP_G32;
           a.row0 = p0;
           a.tile0 = (int)((int64_t)tiles * q / runs);
           a.n_tiles = (int)((int64_t)tiles * (q + 1) / runs) - a.tile0;
-          a.nbc = nbc; a.v_mode = b.v_mode;
+          a.nbc1 = nbc1; a.nbc2 = nbc2; a.v_mode = b.v_mode;
           a.v_group_rows = b.v_group_rows == 0 ? b.rows : b.v_group_rows;
           a.lr_scale = b.lr_scale; a.wd = b.weight_decay;
           items.push_back(a);
         }
       }
     }
-    // shared memory: both factor sets of the L panel, a ring of R^T boxes, a ring of g / W quarter tiles
-    const int l_region = 2 * nbc_max * tc::kBoxBytes;
-    P->apply_r_stages = 2;   // (a deeper R ring measured no faster; the g / W ring is what pays)
+    // shared memory: the L panel (both factor sets side by side), a ring of R^T boxes, a ring of g / W quarter
+    // tiles.  Three R stages, and whatever is left for g / W: measured, the g / W ring pays more per KB than a
+    // deeper R ring, but two R stages leave the MMA warp waiting on every box.
+    const int l_region = nbc_max * tc::kBoxBytes;
+    P->apply_r_stages = 3;
     P->apply_r_region = l_region;
     P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
-    P->apply_bufs = std::max(1, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / tc::kApplyBufBytes));
+    P->apply_bufs = std::max(2, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / tc::kApplyBufBytes));
     P->smem_apply = P->apply_w_region + P->apply_bufs * tc::kApplyBufBytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
              std::min<int64_t>((int64_t)items.size(), P->n_sms)};
@@ -406,11 +421,14 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
     ok = ok && tc::encode_panel32(&m[MAP_W], params + blk.offset * 4, rows, cols, true);
     ok = ok && tc::encode_panel32(&m[MAP_G32], grads + blk.offset * 2, rows, cols, false);
     for (int q = 0; q < 3; ++q) {
-      ok = ok && tc::encode_bf16_matrix(&m[MAP_LC + q], work + t.lc[q] * 2, rows, 2 * rp, 2 * rp);
-      ok = ok && tc::encode_bf16_chunked(&m[MAP_LC_N + q], work + t.lc[q] * 2, rows, 2 * rp, nb, 128);
-      ok = ok && tc::encode_bf16_matrix(&m[MAP_RTC + q], work + t.rtc[q] * 2, cols, 2 * rp, 2 * rp);
-      ok = ok && tc::encode_bf16_chunked(&m[MAP_RTC_N + q], work + t.rtc[q] * 2, cols, 2 * rp, nb, 128);
+      const uint64_t ld = (uint64_t)t.ld[q];
+      ok = ok && tc::encode_bf16_matrix(&m[MAP_LC + q], work + t.lc[q] * 2, rows, 2 * rp, ld);
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_LC_N + q], work + t.lc[q] * 2, rows, ld, nb, 128);
+      ok = ok && tc::encode_bf16_matrix(&m[MAP_RTC + q], work + t.rtc[q] * 2, cols, 2 * rp, ld);
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_RTC_N + q], work + t.rtc[q] * 2, cols, ld, nb, 128);
     }
+    ok = ok && tc::encode_bf16_matrix(&m[MAP_LCAT], work + t.lc[0] * 2, rows, 4 * rp, 4 * rp);
+    ok = ok && tc::encode_bf16_matrix(&m[MAP_RCAT], work + t.rtc[0] * 2, cols, 4 * rp, 4 * rp);
     for (int q = 0; q < 4; ++q)
       ok = ok && tc::encode_bf16_chunked(&m[MAP_GS + q], work + t.gs[q] * 2, rp, 2 * rp, nb, (uint32_t)rp);
     if (!ok) {

@@ -4,12 +4,13 @@
 //   m^c = cg g + c0 L0 R0 - c1 L R          (= g + c (P_{t-1} - P_t) with the correction on)
 //   W  <- W - lr s_b ( clamp( m^c / (sqrt(v) + eps) ) + lambda_b W )
 //
-// An item is a 128-row panel of one block times a run of column tiles.  The split-bf16 rows of L0
-// and L of the panel stay in shared memory for the whole run; per column tile the matching rows of
-// R0^T and R^T arrive one 64-column box at a time through a ring of 16 KB stages, and every box is
-// multiplied at once with the resident L columns it pairs with (hi*hi and lo*hi for a column of the
-// hi half, hi*lo for a column of the lo half; the new pair with a negated A operand), so the
-// accumulator ends up holding D = L0 R0 - L R.
+// An item is a 128-row panel of one block times a run of column tiles.  The split-bf16 rows
+// [L0 hi | L0 lo | L hi | L lo] of the panel stay in shared memory for the whole run; per column tile
+// the matching rows of [R0^T hi | R0^T lo | R^T hi | R^T lo] arrive one 64-column box at a time
+// through a ring of 16 KB stages, and every 16 columns of a box are multiplied at once with the
+// resident L columns they pair with (hi*hi and lo*hi for columns of a hi part, hi*lo for columns of
+// a lo part; the new set with a negated A operand), so the accumulator ends up holding
+// D = L0 R0 - L R.
 //
 // g and W never pass through registers on their way in or out: a mover thread brings them in
 // quarter tiles (128 rows x 32 columns: 16 KB of W, 8 KB of g) by TMA into a small ring of
@@ -42,11 +43,12 @@ struct ApplyItem {
   int64_t off;               // element offset of the block in params / grads
   int64_t v_off;             // float offset of v in state
   int32_t rows, cols, r, rp;
-  int32_t map_l0, map_l1, map_r0, map_r1;   // split factors: [rows, 2rp] and [cols, 2rp], boxes of 64 x 128
+  int32_t map_l, map_r;      // split factors, previous and final set side by side: [rows, 4rp] and [cols, 4rp]
+                             // = [hi0 | lo0 | hi1 | lo1], boxes of 64 x 128
   int32_t map_w, map_g;      // params and grads of the block, boxes of 32 x 128
   int32_t row0;              // first row of the panel
   int32_t tile0, n_tiles;    // column tiles [tile0, tile0 + n_tiles) of 128 columns
-  int32_t nbc;               // 64-wide boxes across the 2rp split columns
+  int32_t nbc1, nbc2;        // 64-wide boxes across the 2rp columns of the previous set / the 4rp of both
   int32_t v_mode, v_group_rows;
   float lr_scale, wd;
 };
@@ -111,24 +113,19 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
         const ApplyItem I = a.items[it];
         if (!mbar_wait(&sh.lempty, item_phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
-        mbar_arrive_expect_tx(&sh.lfull, (uint32_t)(n_sets * I.nbc) * kBoxBytes);
-        for (int set = 0; set < n_sets; ++set) {
-          const CUtensorMap* m = a.maps + (set ? I.map_l1 : I.map_l0);
-          for (int bc = 0; bc < I.nbc; ++bc)
-            tma_load_box(smem_l + (size_t)(set * I.nbc + bc) * kBoxBytes, m, 64 * bc, I.row0, &sh.lfull);
-        }
+        const int nb = n_sets == 2 ? I.nbc2 : I.nbc1;
+        mbar_arrive_expect_tx(&sh.lfull, (uint32_t)nb * kBoxBytes);
+        for (int bc = 0; bc < nb; ++bc)
+          tma_load_box(smem_l + (size_t)bc * kBoxBytes, a.maps + I.map_l, 64 * bc, I.row0, &sh.lfull);
         ++l_loads;
         for (int t = 0; t < I.n_tiles && ok; ++t) {
           const int col0 = (I.tile0 + t) * kApplyNT;
-          for (int set = 0; set < n_sets && ok; ++set) {
-            const CUtensorMap* m = a.maps + (set ? I.map_r1 : I.map_r0);
-            for (int bc = 0; bc < I.nbc; ++bc) {
-              if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
-              mbar_arrive_expect_tx(&sh.rfull[rs], (uint32_t)kBoxBytes);
-              tma_load_box(smem_r + (size_t)rs * kBoxBytes, m, 64 * bc, col0, &sh.rfull[rs]);
-              ++r_loads;
-              if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
-            }
+          for (int bc = 0; bc < nb; ++bc) {
+            if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
+            mbar_arrive_expect_tx(&sh.rfull[rs], (uint32_t)kBoxBytes);
+            tma_load_box(smem_r + (size_t)rs * kBoxBytes, a.maps + I.map_r, 64 * bc, col0, &sh.rfull[rs]);
+            ++r_loads;
+            if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
           }
         }
         item_phase ^= 1u;
@@ -157,7 +154,12 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
       const uint32_t dhi = desc_hi();
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
         const ApplyItem I = a.items[it];
-        const int ks = I.rp >> 4;     // 16-wide K steps per part
+        const int ks = I.rp >> 4;     // 16-wide K steps per part (hi or lo of one set)
+        const int ktot = n_sets * 2 * ks;
+        const int nb = n_sets == 2 ? I.nbc2 : I.nbc1;
+        const uint32_t idesc_pos = make_idesc(kApplyNT, false, false, false);
+        const uint32_t idesc_neg = make_idesc(kApplyNT, false, false, true);
+        const uint32_t la = desc_lo(l_base, 16);
         if (!mbar_wait(&sh.lfull, item_phase, abort, a.status, ST_WAIT_FULL)) break;
         for (int t = 0; t < I.n_tiles && ok; ++t, ++j) {
           const int acc = j & 1;
@@ -165,30 +167,29 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           if (!mbar_wait(&sh.tempty[acc], acc_phase ^ 1u, abort, a.status, ST_WAIT_TMEM_EMPTY)) { ok = false; break; }
           const uint32_t d = tmem_base + (uint32_t)(acc * kApplyNT);
           uint32_t accumulate = 0;
-          // K step k of a [.., 2rp] operand: box k / 4 (16 KB apart), 32 bytes per step inside it
+          // K step k of the [.., 4rp] operands: box k / 4 (16 KB apart), 32 bytes per step inside it
           auto kstep = [](int k) { return (uint32_t)((k >> 2) * (kBoxBytes >> 4) + (k & 3) * 2); };
-          for (int set = 0; set < n_sets && ok; ++set) {
-            const uint32_t idesc = make_idesc(kApplyNT, false, false, set == 1);
-            const uint32_t la = desc_lo(l_base + (uint32_t)(set * I.nbc) * kBoxBytes, 16);
-            for (int bc = 0; bc < I.nbc; ++bc) {
-              if (!mbar_wait(&sh.rfull[rs], rphase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
-              tc_fence_after();
-              const uint32_t rb = desc_lo(r_base + (uint32_t)rs * kBoxBytes, 16);
-              for (int kk = 0; kk < 4; ++kk) {
-                const int kb = 4 * bc + kk;            // K step of [R hi | R lo] held by this box
-                if (kb >= 2 * ks) break;
-                const uint64_t b = desc_join(rb + (uint32_t)(kk * 2), dhi);
-                if (kb < ks) {                         // hi * hi, lo * hi
-                  mma_bf16(d, desc_join(la + kstep(kb), dhi), b, idesc, accumulate);
-                  mma_bf16(d, desc_join(la + kstep(ks + kb), dhi), b, idesc, 1u);
-                } else {                               // hi * lo
-                  mma_bf16(d, desc_join(la + kstep(kb - ks), dhi), b, idesc, accumulate);
-                }
-                accumulate = 1;
+          for (int bc = 0; bc < nb; ++bc) {
+            if (!mbar_wait(&sh.rfull[rs], rphase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t rb = desc_lo(r_base + (uint32_t)rs * kBoxBytes, 16);
+            for (int kk = 0; kk < 4; ++kk) {
+              const int kb = 4 * bc + kk;              // K step of [R0 hi | R0 lo | R hi | R lo] held by this box
+              if (kb >= ktot) break;
+              const int set = kb >= 2 * ks ? 1 : 0;
+              const int w = kb - set * 2 * ks;         // K step inside the set: hi part, then lo part
+              const uint32_t idesc = set ? idesc_neg : idesc_pos;
+              const uint64_t b = desc_join(rb + (uint32_t)(kk * 2), dhi);
+              if (w < ks) {                            // hi * hi, lo * hi
+                mma_bf16(d, desc_join(la + kstep(kb), dhi), b, idesc, accumulate);
+                mma_bf16(d, desc_join(la + kstep(kb + ks), dhi), b, idesc, 1u);
+              } else {                                 // hi * lo
+                mma_bf16(d, desc_join(la + kstep(kb - ks), dhi), b, idesc, accumulate);
               }
-              mma_commit(&sh.rempty[rs]);
-              if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
+              accumulate = 1;
             }
+            mma_commit(&sh.rempty[rs]);
+            if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
           }
           if (ok) mma_commit(&sh.tfull[acc]);
         }
