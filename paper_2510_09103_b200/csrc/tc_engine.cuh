@@ -282,7 +282,19 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       // old values travel one piece ahead in two register sets that swap roles (no copies, which
       // would wait for the loads); the first set is requested before the accumulator is waited for
       float oldA[4][4], oldB[4][4];
-      if (factor) fetch_old(0, oldA);
+      // A factor whose consecutive owners are adjacent in memory (R, stored [r, n]) needs no turn: for
+      // a fixed column the 32 rows of a warp are one 128-byte run already.  Old values of this
+      // thread's own row, columns [p, p+16), kept in the same registers as o[e / 4][e % 4].
+      const bool by_column = factor && I.own_stride == 1 && !vec4;
+      const int own_row = (second ? I.own1 : I.own0) + q;
+      auto fetch_old_col = [&](int p, float (*o)[4]) {
+        const float* fp = fbase + own_row + I.k_stride * p;
+        const bool row_ok = own_row < I.own_count;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e >> 2][e & 3] = (row_ok && p + e < r) ? __ldcg(fp + I.k_stride * e) : 0.f;
+      };
+      if (by_column) fetch_old_col(0, oldA);
+      else if (factor) fetch_old(0, oldA);
       // one lane per warp polls (fewer pollers on the barrier), then the warp agrees: the
       // tensor-memory loads below need all 32 lanes
       bool got = true;
@@ -361,13 +373,50 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             *reinterpret_cast<uint2*>(drow + rp) = make_uint2(l01, l23);
           }
         };
+        // the same piece without the turn: this thread's row, columns [p, p+16)
+        auto piece_col = [&](int p, float (*o)[4]) {
+          float d0[16], d1[16];
+          tmem_ld16(t0 + (uint32_t)p, d0);
+          tmem_ld16(t0 + (uint32_t)(rp + p), d1);
+          tmem_ld_wait();
+          if (own_row >= I.own_count) return;
+          float* fp = fbase + own_row + I.k_stride * p;
+          uint32_t hi[8], lo[8];
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            const float x0 = p + e < r ? o[e >> 2][e & 3] + I.coef * (d0[e] + d1[e]) : 0.f;
+            const float x1 = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * (d0[e + 1] + d1[e + 1]) : 0.f;
+            if (p + e < r) fp[I.k_stride * e] = x0;
+            if (p + e + 1 < r) fp[I.k_stride * (e + 1)] = x1;
+            split_bf16x2(x0, x1, hi[e >> 1], lo[e >> 1]);
+          }
+          uint16_t* drow = dst + (int64_t)I.dst_ld * own_row + p;
+          uint4* dh = reinterpret_cast<uint4*>(drow);
+          uint4* dl = reinterpret_cast<uint4*>(drow + rp);
+          dh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          dh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+          dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        };
+        if (by_column) {
 #pragma unroll 1
-        for (int p = 0; p < rp; p += 32) {
-          if (p + 16 < rp) fetch_old(p + 16, oldB);
-          piece(p, oldA);
-          if (p + 16 < rp) {
-            if (p + 32 < rp) fetch_old(p + 32, oldA);
-            piece(p + 16, oldB);
+          for (int p = 0; p < rp; p += 32) {
+            if (p + 16 < rp) fetch_old_col(p + 16, oldB);
+            piece_col(p, oldA);
+            if (p + 16 < rp) {
+              if (p + 32 < rp) fetch_old_col(p + 32, oldA);
+              piece_col(p + 16, oldB);
+            }
+          }
+        } else {
+#pragma unroll 1
+          for (int p = 0; p < rp; p += 32) {
+            if (p + 16 < rp) fetch_old(p + 16, oldB);
+            piece(p, oldA);
+            if (p + 16 < rp) {
+              if (p + 32 < rp) fetch_old(p + 32, oldA);
+              piece(p + 16, oldB);
+            }
           }
         }
       } else if (I.epi == EPI_GRAM) {
