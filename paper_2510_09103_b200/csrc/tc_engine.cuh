@@ -293,7 +293,24 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
 #pragma unroll
         for (int e = 0; e < 16; ++e) o[e >> 2][e & 3] = (row_ok && p + e < r) ? __ldcg(fp + I.k_stride * e) : 0.f;
       };
-      if (by_column) fetch_old_col(0, oldA);
+      // A factor stored row by row (L, [m, r]) whose rows start on 32-byte boundaries and hold a multiple of
+      // eight values needs no turn either: a lane moves 32 bytes per access, which is a whole sector.
+      const bool by_row = factor && I.k_stride == 1 && ((I.own_stride | r | I.f32_off) & 7) == 0;
+      auto fetch_old_row = [&](int p, float (*o)[4]) {
+        const float* fp = fbase + I.own_stride * own_row + p;
+        const bool row_ok = own_row < I.own_count;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (row_ok && p + 8 * h < r) {
+            ldcg_f32x8(fp + 8 * h, &o[2 * h][0]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[2 * h + (e >> 2)][e & 3] = 0.f;
+          }
+        }
+      };
+      if (by_row) fetch_old_row(0, oldA);
+      else if (by_column) fetch_old_col(0, oldA);
       else if (factor) fetch_old(0, oldA);
       // one lane per warp polls (fewer pollers on the barrier), then the warp agrees: the
       // tensor-memory loads below need all 32 lanes
@@ -398,7 +415,39 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
           dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
         };
-        if (by_column) {
+        // and for a row-stored factor with aligned rows
+        auto piece_row = [&](int p, float (*o)[4]) {
+          float d0[16], d1[16];
+          tmem_ld16(t0 + (uint32_t)p, d0);
+          tmem_ld16(t0 + (uint32_t)(rp + p), d1);
+          tmem_ld_wait();
+          if (own_row >= I.own_count) return;
+          float x[16];
+          uint32_t hi[8], lo[8];
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            x[e] = p + e < r ? o[e >> 2][e & 3] + I.coef * (d0[e] + d1[e]) : 0.f;
+            x[e + 1] = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * (d0[e + 1] + d1[e + 1]) : 0.f;
+            split_bf16x2(x[e], x[e + 1], hi[e >> 1], lo[e >> 1]);
+          }
+          float* fp = fbase + I.own_stride * own_row + p;
+          if (p < r) st_f32x8(fp, x);
+          if (p + 8 < r) st_f32x8(fp + 8, x + 8);
+          uint16_t* drow = dst + (int64_t)I.dst_ld * own_row + p;
+          st_b32x8(drow, hi);
+          st_b32x8(drow + rp, lo);
+        };
+        if (by_row) {
+#pragma unroll 1
+          for (int p = 0; p < rp; p += 32) {
+            if (p + 16 < rp) fetch_old_row(p + 16, oldB);
+            piece_row(p, oldA);
+            if (p + 16 < rp) {
+              if (p + 32 < rp) fetch_old_row(p + 32, oldA);
+              piece_row(p + 16, oldB);
+            }
+          }
+        } else if (by_column) {
 #pragma unroll 1
           for (int p = 0; p < rp; p += 32) {
             if (p + 16 < rp) fetch_old_col(p + 16, oldB);
