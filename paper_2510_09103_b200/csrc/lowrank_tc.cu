@@ -29,10 +29,10 @@ namespace {
 
 // tensor maps of one block: g; Lc[3] and RTc[3] each as a plain matrix (A side) and as 64-column
 // chunks (N side); Gs[4] as chunks; W and g in quarter-tile boxes; the previous and the final set of
-// Lc and of RTc side by side as one matrix (the apply kernel's operands)
-constexpr int kMapsPerBlock = 21;
+// Lc and of RTc side by side as one matrix (the apply kernel's operands); a per-element v like W
+constexpr int kMapsPerBlock = 22;
 enum { MAP_G = 0, MAP_LC = 1, MAP_LC_N = 4, MAP_RTC = 7, MAP_RTC_N = 10, MAP_GS = 13, MAP_W = 17, MAP_G32 = 18,
-       MAP_LCAT = 19, MAP_RCAT = 20 };
+       MAP_LCAT = 19, MAP_RCAT = 20, MAP_V = 21 };
 
 struct ConvertJob {
   int64_t f32_off;          // float offset of the factor in state
@@ -101,7 +101,7 @@ struct TcProgram {
     e.smem = e.n_stages * e.stage_bytes + 1024;
     return e;
   }
-  int apply_r_region = 0, apply_r_stages = 3, apply_w_region = 0, apply_bufs = 2;
+  int apply_r_region = 0, apply_r_stages = 3, apply_w_region = 0, apply_bufs = 2, apply_buf_bytes = 0;
   int n_sms = 148;
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
@@ -110,6 +110,7 @@ struct TcProgram {
   const void* enc_grads = nullptr;
   const void* enc_work = nullptr;
   const void* enc_params = nullptr;
+  const void* enc_state = nullptr;
   cudaEvent_t maps_copied = nullptr;
 };
 
@@ -340,12 +341,14 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
   {
     std::vector<tc::ApplyItem> items;
     int nbc_max = 1;
+    bool any_element_v = false;
     for (size_t bi = 0; bi < P->blk.size(); ++bi) {
       const TcBlock& t = P->blk[bi];
       const adapm_block& b = c->blocks[t.id];
       const int mb = (int)bi * kMapsPerBlock;
       const int nbc1 = (2 * t.rp + 63) / 64, nbc2 = (4 * t.rp + 63) / 64;
       nbc_max = std::max(nbc_max, nbc2);
+      if (b.v_mode == ADAPM_V_ELEMENT) any_element_v = true;
       const int tiles = (b.cols + tc::kApplyNT - 1) / tc::kApplyNT;
       const int runs = (tiles + 15) / 16;
       for (int p0 = 0; p0 < b.rows; p0 += 128) {
@@ -354,7 +357,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           std::memset(&a, 0, sizeof(a));
           a.off = b.offset; a.v_off = c->v_off[t.id]; a.rows = b.rows; a.cols = b.cols; a.r = b.rank; a.rp = t.rp;
           a.map_l = mb + MAP_LCAT; a.map_r = mb + MAP_RCAT;
-          a.map_w = mb + MAP_W; a.map_g = mb + MAP_G32;
+          a.map_w = mb + MAP_W; a.map_g = mb + MAP_G32; a.map_v = mb + MAP_V;
           a.row0 = p0;
           a.tile0 = (int)((int64_t)tiles * q / runs);
           a.n_tiles = (int)((int64_t)tiles * (q + 1) / runs) - a.tile0;
@@ -372,8 +375,13 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     P->apply_r_stages = 3;
     P->apply_r_region = l_region;
     P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
-    P->apply_bufs = std::max(2, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / tc::kApplyBufBytes));
-    P->smem_apply = P->apply_w_region + P->apply_bufs * tc::kApplyBufBytes + 1024;
+    P->apply_buf_bytes = tc::kApplyBufBytes + (any_element_v ? tc::kWBoxBytes : 0);
+    if (226 * 1024 - P->apply_w_region < 2 * P->apply_buf_bytes) {   // two buffers at least: give up R stages
+      P->apply_r_stages = 2;
+      P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
+    }
+    P->apply_bufs = std::max(1, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / P->apply_buf_bytes));
+    P->smem_apply = P->apply_w_region + P->apply_bufs * P->apply_buf_bytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
              std::min<int64_t>((int64_t)items.size(), P->n_sms)};
     prog.push_back(A);
@@ -399,18 +407,21 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
 // per-step work
 // ---------------------------------------------------------------------------------------------------
 
-// Tensor maps hold absolute addresses: (re)build them when the parameter, gradient or workspace buffer moved.
+// Tensor maps hold absolute addresses: (re)build them when the parameter, gradient, state or workspace buffer
+// moved.
 // The copy to the device is asynchronous on `s`; only a second move while that copy is still in
 // flight waits for it (the staging buffer is reused).
 int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
   TcProgram* P = c->tc;
   if (!P || P->blk.empty()) return ADAPM_OK;
-  if (P->enc_grads == b.p[BASE_GRADS] && P->enc_work == b.p[BASE_WORK] && P->enc_params == b.p[BASE_PARAMS])
+  if (P->enc_grads == b.p[BASE_GRADS] && P->enc_work == b.p[BASE_WORK] && P->enc_params == b.p[BASE_PARAMS] &&
+      P->enc_state == b.p[BASE_STATE])
     return ADAPM_OK;
   if (P->enc_grads) ADAPM_CUDA(cudaEventSynchronize(P->maps_copied));
   const char* grads = static_cast<const char*>(b.p[BASE_GRADS]);
   const char* work = static_cast<const char*>(b.p[BASE_WORK]);
   const char* params = static_cast<const char*>(b.p[BASE_PARAMS]);
+  const char* state = static_cast<const char*>(b.p[BASE_STATE]);
   for (size_t bi = 0; bi < P->blk.size(); ++bi) {
     const TcBlock& t = P->blk[bi];
     const adapm_block& blk = c->blocks[t.id];
@@ -420,6 +431,10 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
     bool ok = tc::encode_bf16_matrix(&m[MAP_G], grads + blk.offset * 2, rows, cols, cols);
     ok = ok && tc::encode_panel32(&m[MAP_W], params + blk.offset * 4, rows, cols, true);
     ok = ok && tc::encode_panel32(&m[MAP_G32], grads + blk.offset * 2, rows, cols, false);
+    if (blk.v_mode == ADAPM_V_ELEMENT)
+      ok = ok && tc::encode_panel32(&m[MAP_V], state + c->v_off[t.id] * 4, rows, cols, true);
+    else
+      std::memset(&m[MAP_V], 0, sizeof(CUtensorMap));
     for (int q = 0; q < 3; ++q) {
       const uint64_t ld = (uint64_t)t.ld[q];
       ok = ok && tc::encode_bf16_matrix(&m[MAP_LC + q], work + t.lc[q] * 2, rows, 2 * rp, ld);
@@ -442,6 +457,7 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s) {
   P->enc_grads = b.p[BASE_GRADS];
   P->enc_work = b.p[BASE_WORK];
   P->enc_params = b.p[BASE_PARAMS];
+  P->enc_state = b.p[BASE_STATE];
   return ADAPM_OK;
 }
 
@@ -472,7 +488,7 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.state = (float*)b.p[BASE_STATE]; a.status = c->d_status; a.sc = sc;
       a.use_new = sc.c1 != 0.f ? 1 : 0;
       a.r_region_off = P->apply_r_region; a.n_rstages = P->apply_r_stages;
-      a.w_region_off = P->apply_w_region; a.n_bufs = P->apply_bufs;
+      a.w_region_off = P->apply_w_region; a.n_bufs = P->apply_bufs; a.buf_bytes = P->apply_buf_bytes;
       tc::tc_apply_kernel<<<(unsigned)L.grid, tc::kApplyThreads, P->smem_apply, s>>>(a);
       break;
     }

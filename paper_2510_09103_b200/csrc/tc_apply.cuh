@@ -17,8 +17,8 @@
 // shared-memory buffers, several quarters ahead of their use, and writes the updated W back from
 // the same buffer by TMA.  Each of the 256 epilogue threads owns one row of the panel: it reads its
 // accumulator row from tensor memory, its 16 columns of g and W from the (swizzled) buffer, and
-// puts the new W back in place.  Only a per-element v, where a block has one, is read and written
-// directly.  The m x n matrices m_t, r_t and m^c are never stored.
+// puts the new W back in place.  A per-element v, where a block has one, travels like W.
+// The m x n matrices m_t, r_t and m^c are never stored.
 #pragma once
 
 #include <cuda.h>
@@ -37,7 +37,7 @@ constexpr int kApplyMaxStages = 8;         // R ring depth limit
 constexpr int kApplyMaxBufs = 6;           // g / W ring depth limit
 constexpr int kWBoxBytes = 128 * kApplyQC * 4;   // a quarter tile of W: 128 rows of 128 bytes
 constexpr int kGBoxBytes = 128 * kApplyQC * 2;   // and of g: 128 rows of 64 bytes
-constexpr int kApplyBufBytes = kWBoxBytes + kGBoxBytes;
+constexpr int kApplyBufBytes = kWBoxBytes + kGBoxBytes;    // + kWBoxBytes where a block has a per-element v
 
 struct ApplyItem {
   int64_t off;               // element offset of the block in params / grads
@@ -46,6 +46,7 @@ struct ApplyItem {
   int32_t map_l, map_r;      // split factors, previous and final set side by side: [rows, 4rp] and [cols, 4rp]
                              // = [hi0 | lo0 | hi1 | lo1], boxes of 64 x 128
   int32_t map_w, map_g;      // params and grads of the block, boxes of 32 x 128
+  int32_t map_v;             // per-element v of the block (same boxes as params); unused with a group v
   int32_t row0;              // first row of the panel
   int32_t tile0, n_tiles;    // column tiles [tile0, tile0 + n_tiles) of 128 columns
   int32_t nbc1, nbc2;        // 64-wide boxes across the 2rp columns of the previous set / the 4rp of both
@@ -64,7 +65,8 @@ struct ApplyArgs {
   int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
   int32_t n_rstages;         // R ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
   int32_t w_region_off;      // byte offset of the g / W ring
-  int32_t n_bufs;            // g / W ring depth (1..kApplyMaxBufs); a buffer is kApplyBufBytes
+  int32_t n_bufs;            // g / W ring depth (1..kApplyMaxBufs)
+  int32_t buf_bytes;         // one buffer: W, g and, if any block of the launch has a per-element v, v
 };
 
 struct __align__(8) ApplyShared {
@@ -206,11 +208,13 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
       if (ld_it < a.n_items) { LI = a.items[ld_it]; ld_nq = 4 * LI.n_tiles; }
       auto load_next = [&]() {
         const int b = n_loaded % a.n_bufs;
-        uint8_t* buf = smem_w + (size_t)b * kApplyBufBytes;
+        uint8_t* buf = smem_w + (size_t)b * a.buf_bytes;
         const int col = (LI.tile0 + (ld_q >> 2)) * kApplyNT + (ld_q & 3) * kApplyQC;
-        mbar_arrive_expect_tx(&sh.wfull[b], (uint32_t)kApplyBufBytes);
+        const bool with_v = LI.v_mode == ADAPM_V_ELEMENT;
+        mbar_arrive_expect_tx(&sh.wfull[b], (uint32_t)(kApplyBufBytes + (with_v ? kWBoxBytes : 0)));
         tma_load_box(buf, a.maps + LI.map_w, col, LI.row0, &sh.wfull[b]);
         tma_load_box(buf + kWBoxBytes, a.maps + LI.map_g, col, LI.row0, &sh.wfull[b]);
+        if (with_v) tma_load_box(buf + kApplyBufBytes, a.maps + LI.map_v, col, LI.row0, &sh.wfull[b]);
         ++n_loaded;
         if (++ld_q == ld_nq) {
           ld_it += gridDim.x; ld_q = 0; ld_nq = 0;
@@ -227,15 +231,19 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           if (!mbar_wait(&sh.wdone[b], (uint32_t)(k / a.n_bufs) & 1u, abort, a.status, ST_WAIT_DRAIN)) { ok = false; break; }
           const int col = (I.tile0 + (q >> 2)) * kApplyNT + (q & 3) * kApplyQC;
           // (a quarter that lies past the last column is not stored)
-          if (col < I.cols) tma_store_box(a.maps + I.map_w, col, I.row0, smem_w + (size_t)b * kApplyBufBytes);
+          if (col < I.cols) {
+            const uint8_t* buf = smem_w + (size_t)b * a.buf_bytes;
+            tma_store_box(a.maps + I.map_w, col, I.row0, buf);
+            if (I.v_mode == ADAPM_V_ELEMENT) tma_store_box(a.maps + I.map_v, col, I.row0, buf + kApplyBufBytes);
+          }
           bulk_commit_group();
-          if ((k & 1) && ld_it < a.n_items) {
+          if ((a.n_bufs < 2 || (k & 1)) && ld_it < a.n_items) {
             // two quarters at a time: their rows are neighbours in memory, and requests that reach DRAM
             // together share its open pages.  They go into this buffer and the one stored before it,
             // once both stores have read them.
             bulk_wait_group_read<0>();
             load_next();
-            if (ld_it < a.n_items) load_next();
+            if (a.n_bufs >= 2 && ld_it < a.n_items) load_next();
           }
         }
       }
@@ -275,23 +283,11 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
       // one denominator per row when v is a group scalar: m^c / (sqrt(v) + eps) becomes a product
       const float v_row = (rok && grouped) ? a.state[I.v_off + row / I.v_group_rows] : 0.f;
       const float kr = sc.inv_bc1 / (sqrtf(v_row * sc.inv_bc2) + sc.eps);
-      float* vrow = a.state + I.v_off + (int64_t)row * I.cols;   // per-element v of this row (not grouped)
       const int n_q = 4 * I.n_tiles;
-      auto v_col = [&](int q) { return (I.tile0 + (q >> 2)) * kApplyNT + (q & 3) * kApplyQC + 16 * half; };
-      auto v_fetch = [&](int q, float4* v) {
-        const int col = v_col(q);
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          v[i] = (rok && col + 4 * i + 4 <= I.cols) ? __ldcg(reinterpret_cast<const float4*>(vrow + col) + i)
-                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-      };
-      float4 vq[4], vn[4];
-      if (!grouped) v_fetch(0, vq);
       for (int q = 0; q < n_q; ++q, ++k) {
         const int jt = j + (q >> 2), sub = q & 3;
         const int acc = jt & 1;
         const int b = k % a.n_bufs;
-        if (!grouped && q + 1 < n_q) v_fetch(q + 1, vn);
         if (sub == 0) {
           // one lane per warp polls, then the warp agrees: the tensor-memory loads need all 32 lanes
           bool got = true;
@@ -306,7 +302,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
         ok = __all_sync(0xffffffffu, ok);
         tmem_ld_wait();
         if (!ok) break;
-        uint8_t* buf = smem_w + (size_t)b * kApplyBufBytes;
+        uint8_t* buf = smem_w + (size_t)b * a.buf_bytes;
         float gf[16];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -318,7 +314,6 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
             gf[8 * i + 2 * x + 1] = __uint_as_float(gw[x] & 0xffff0000u);
           }
         }
-        const int col = v_col(q);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float4* wp = reinterpret_cast<float4*>(buf + w_at[i]);
@@ -332,15 +327,16 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
               w[x] = w[x] - lr_s * (ratio + I.wd * w[x]);
             }
           } else {
-            float vv[4] = {vq[i].x, vq[i].y, vq[i].z, vq[i].w};
+            float4* vp = reinterpret_cast<float4*>(buf + kApplyBufBytes + w_at[i]);   // v lies like W
+            const float4 vo = *vp;
+            float vv[4] = {vo.x, vo.y, vo.z, vo.w};
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
               const float g1 = gf[4 * i + x];
               vv[x] = sc.beta2 * vv[x] + (1.f - sc.beta2) * (g1 * g1);
               w[x] = adapm_param_update(w[x], sc.cg * g1 + sc.c0 * d[4 * i + x], vv[x], sc, lr_s, I.wd);
             }
-            if (rok && col + 4 * i + 4 <= I.cols)
-              *(reinterpret_cast<float4*>(vrow + col) + i) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+            *vp = make_float4(vv[0], vv[1], vv[2], vv[3]);
           }
           *wp = make_float4(w[0], w[1], w[2], w[3]);
         }
@@ -351,10 +347,6 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
         if (lane == 0) {
           mbar_arrive(&sh.wdone[b]);
           if (sub == 3) mbar_arrive(&sh.tempty[acc]);
-        }
-        if (!grouped) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) vq[i] = vn[i];
         }
       }
       j += I.n_tiles;

@@ -408,12 +408,8 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             split_bf16x2(x0, x1, hi[e >> 1], lo[e >> 1]);
           }
           uint16_t* drow = dst + (int64_t)I.dst_ld * own_row + p;
-          uint4* dh = reinterpret_cast<uint4*>(drow);
-          uint4* dl = reinterpret_cast<uint4*>(drow + rp);
-          dh[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          dh[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-          dl[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-          dl[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+          st_b32x8(drow, hi);
+          st_b32x8(drow + rp, lo);
         };
         // and for a row-stored factor with aligned rows
         auto piece_row = [&](int p, float (*o)[4]) {
