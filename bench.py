@@ -44,7 +44,7 @@ def _peaks():
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload
 # (profiles/ holds the captures these come from).  tc_panel: captured on the 4-layer case gpt2_1p5b@4
 # (446.4 MB per launch) and scaled by 12, since every low-rank block belongs to a layer.
-NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 12 * 446.4e6}
+NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 12 * 492.9e6}
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
