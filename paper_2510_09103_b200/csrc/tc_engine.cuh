@@ -403,8 +403,8 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           for (int e = 0; e < 16; e += 2) {
             const float x0 = p + e < r ? o[e >> 2][e & 3] + I.coef * (d0[e] + d1[e]) : 0.f;
             const float x1 = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * (d0[e + 1] + d1[e + 1]) : 0.f;
-            if (p + e < r) fp[I.k_stride * e] = x0;
-            if (p + e + 1 < r) fp[I.k_stride * (e + 1)] = x1;
+            if (p + e < r) __stcg(fp + I.k_stride * e, x0);
+            if (p + e + 1 < r) __stcg(fp + I.k_stride * (e + 1), x1);
             split_bf16x2(x0, x1, hi[e >> 1], lo[e >> 1]);
           }
           uint16_t* drow = dst + (int64_t)I.dst_ld * own_row + p;
