@@ -136,7 +136,7 @@ struct Launch {
   int64_t table_off;    // byte offset of its descriptor table in the device table blob
   int64_t n_items;      // descriptors
   int64_t grid;         // CTAs
-  int64_t aux0 = 0, aux1 = 0, aux2 = 0;
+  int64_t aux0 = 0, aux1 = 0, aux2 = 0, aux3 = 0;
 };
 
 // ---------------------------------------------------------------------------------------------

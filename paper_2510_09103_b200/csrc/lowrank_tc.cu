@@ -173,9 +173,26 @@ int item_cost(const tc::Item& it) {
   return c + 2;   // the epilogue
 }
 
-void sort_by_cost(std::vector<tc::Item>& v) {
+// Hands the items to `grid` CTAs, longest first, each to the CTA with the least work so far.  Afterwards CTA c owns
+// v[begin[c] .. begin[c + 1]).
+void schedule_items(std::vector<tc::Item>& v, int grid, std::vector<int32_t>& begin) {
   for (auto& it : v) it.cost = item_cost(it);
   std::stable_sort(v.begin(), v.end(), [](const tc::Item& a, const tc::Item& b) { return a.cost > b.cost; });
+  std::vector<std::vector<tc::Item>> per(grid);
+  std::vector<int64_t> load(grid, 0);
+  for (const tc::Item& it : v) {
+    int best = 0;
+    for (int c = 1; c < grid; ++c)
+      if (load[c] < load[best]) best = c;
+    per[best].push_back(it);
+    load[best] += it.cost;
+  }
+  v.clear();
+  begin.assign(grid + 1, 0);
+  for (int c = 0; c < grid; ++c) {
+    v.insert(v.end(), per[c].begin(), per[c].end());
+    begin[c + 1] = (int32_t)v.size();
+  }
 }
 
 }  // namespace
@@ -323,16 +340,21 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       for (int p0 = 0; p0 < m; p0 += step) panel(true, p0, pair_panels && p0 + 128 < m);
       for (int p0 = 0; p0 < n; p0 += step) panel(false, p0, pair_panels && p0 + 128 < n);
     }
-    sort_by_cost(grams);
-    sort_by_cost(panels);
-    Launch G{LK_TC_GRAM, append_items(c->h_tables, grams), (int64_t)grams.size(),
-             std::min<int64_t>((int64_t)grams.size(), P->n_sms)};
+    // (Keeping a block's row and column panels together in time, so that their two reads of g share L2, was
+    // measured no faster than plain longest-first: the main loop is not bound by DRAM.)
+    const int grid_g = (int)std::min<int64_t>((int64_t)grams.size(), P->n_sms);
+    const int grid_p = (int)std::min<int64_t>((int64_t)panels.size(), P->n_sms);
+    std::vector<int32_t> begin_g, begin_p;
+    schedule_items(grams, grid_g, begin_g);
+    schedule_items(panels, grid_p, begin_p);
+    Launch G{LK_TC_GRAM, append_items(c->h_tables, grams), (int64_t)grams.size(), grid_g};
     G.aux0 = 4 * rp_max; G.aux1 = 8 * rp_max <= 512 ? 2 : 1; G.aux2 = two_a ? 1 : 0;
+    G.aux3 = append_items(c->h_tables, begin_g);
     prog.push_back(G);
-    Launch Q{LK_TC_PANEL, append_items(c->h_tables, panels), (int64_t)panels.size(),
-             std::min<int64_t>((int64_t)panels.size(), P->n_sms)};
+    Launch Q{LK_TC_PANEL, append_items(c->h_tables, panels), (int64_t)panels.size(), grid_p};
     Q.aux0 = (pair_panels ? 4 : 2) * rp_max; Q.aux1 = (pair_panels ? 8 : 4) * rp_max <= 512 ? 2 : 1;
     Q.aux2 = pair_panels ? 1 : 0;
+    Q.aux3 = append_items(c->h_tables, begin_p);
     prog.push_back(Q);
     src = dst;
   }
@@ -479,6 +501,7 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       const TcProgram::EngineConfig e = P->engine_config(L.aux2 != 0);
       a.stage_bytes = e.stage_bytes; a.n_stages = e.n_stages; a.a_bytes = e.a_bytes;
       a.acc_cols = (int32_t)L.aux0; a.n_acc = (int32_t)L.aux1;
+      a.cta_begin = (const int32_t*)(c->d_tables + L.aux3);
       tc::tc_items_kernel<<<(unsigned)L.grid, tc::kEngineThreads, e.smem, s>>>(a);
       break;
     }

@@ -104,6 +104,7 @@ struct EngineArgs {
   int32_t n_stages;
   int32_t acc_cols;          // tensor-memory columns per accumulator buffer
   int32_t n_acc;             // 1 or 2 accumulator buffers
+  const int32_t* cta_begin;  // CTA c runs items [cta_begin[c], cta_begin[c + 1]) in order
 };
 
 struct __align__(8) EngineShared {
@@ -135,6 +136,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = sh.tmem_base;
+  const int it_begin = a.cta_begin[blockIdx.x], it_end = a.cta_begin[blockIdx.x + 1];
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       uint32_t phase = 0;
       uint32_t issued = 0;
       bool ok = true;
-      for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
+      for (int it = it_begin; it < it_end && ok; ++it) {
         const Item& I = a.items[it];
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const Seg S = I.seg[s];
@@ -191,7 +193,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       int j = 0;
       const uint32_t stages_u32 = smem_u32(stages);
       const uint32_t dhi = desc_hi();
-      for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x, ++j) {
+      for (int it = it_begin; it < it_end && ok; ++it, ++j) {
         const Item& I = a.items[it];
         const int acc = j % a.n_acc;
         const uint32_t acc_phase = (uint32_t)(j / a.n_acc) & 1u;
@@ -239,7 +241,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
     const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
     const bool second = warp >= 6;                      // this warp drains the second accumulator
     int j = 0;
-    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++j) {
+    for (int it = it_begin; it < it_end; ++it, ++j) {
       // scalar fields are copied once: the stores below could alias the item table as far as the
       // compiler can tell, and every re-read would be a round trip to global memory
       ItemEpi I;
