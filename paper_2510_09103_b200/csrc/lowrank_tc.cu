@@ -340,8 +340,9 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       for (int p0 = 0; p0 < m; p0 += step) panel(true, p0, pair_panels && p0 + 128 < m);
       for (int p0 = 0; p0 < n; p0 += step) panel(false, p0, pair_panels && p0 + 128 < n);
     }
-    // (Keeping a block's row and column panels together in time, so that their two reads of g share L2, was
-    // measured no faster than plain longest-first: the main loop is not bound by DRAM.)
+    // (Two schedules that keep a block's row and column panels together in time, so that their two reads of g
+    // could meet in L2 - block order, and teams of CTAs sweeping one block at a time - measured no faster than
+    // longest-first.)
     const int grid_g = (int)std::min<int64_t>((int64_t)grams.size(), P->n_sms);
     const int grid_p = (int)std::min<int64_t>((int64_t)panels.size(), P->n_sms);
     std::vector<int32_t> begin_g, begin_p;
@@ -502,6 +503,9 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.stage_bytes = e.stage_bytes; a.n_stages = e.n_stages; a.a_bytes = e.a_bytes;
       a.acc_cols = (int32_t)L.aux0; a.n_acc = (int32_t)L.aux1;
       a.cta_begin = (const int32_t*)(c->d_tables + L.aux3);
+      // one accumulator buffer of paired panels (4 rp_max columns) leaves room to park their sums (2 rp_max)
+      a.sum_col = (L.kind == LK_TC_PANEL && L.aux2 != 0 && a.n_acc == 1 && a.acc_cols + a.acc_cols / 2 <= 512)
+                      ? a.acc_cols : -1;
       tc::tc_items_kernel<<<(unsigned)L.grid, tc::kEngineThreads, e.smem, s>>>(a);
       break;
     }

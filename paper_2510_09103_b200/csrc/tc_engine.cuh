@@ -105,6 +105,7 @@ struct EngineArgs {
   int32_t acc_cols;          // tensor-memory columns per accumulator buffer
   int32_t n_acc;             // 1 or 2 accumulator buffers
   const int32_t* cta_begin;  // CTA c runs items [cta_begin[c], cta_begin[c + 1]) in order
+  int32_t sum_col;           // EPI_FACTOR: first of the tensor-memory columns the epilogue parks D0 + D1 in, or -1
 };
 
 struct __align__(8) EngineShared {
@@ -322,21 +323,56 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       if (!got) break;
       tc_fence_after();
       const uint32_t t0 = tmem_base + lane_addr + (uint32_t)(acc * a.acc_cols + (second ? I.col2 : 0));
-      if (!has_work) {
-        // nothing to drain for this warp; it still takes part in the hand-back below
-      } else if (I.epi == EPI_FACTOR) {
-        uint16_t* dst = a.work_bf16 + I.dst_off;
-        // one piece: accumulator columns [p, p+16) of this thread's row, old values in `o`
-        auto piece = [&](int p, float (*o)[4]) {
+      // With one accumulator buffer the next item's MMAs wait for this epilogue.  Its memory traffic is the slow
+      // part, so the sums D0 + D1 are first parked in spare tensor-memory columns (this warp's own lanes, the
+      // same columns for every item) and the accumulator is handed back at once; the pieces below then read the
+      // parked sums while the next main loop runs.
+      const bool parked = factor && a.sum_col >= 0;
+      const uint32_t ts = tmem_base + lane_addr + (uint32_t)(a.sum_col + (second ? rp : 0));
+      if (parked) {
+        for (int p = 0; p < rp; p += 16) {
           float d0[16], d1[16];
           tmem_ld16(t0 + (uint32_t)p, d0);
           tmem_ld16(t0 + (uint32_t)(rp + p), d1);
           tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) d0[e] += d1[e];
+          tmem_st16(ts + (uint32_t)p, d0);
+        }
+        tmem_st_wait();
+      }
+      const bool early = parked || !has_work;   // (a warp without work never reads the accumulator)
+      if (early) {
+        tc_fence_before();
+        mbar_arrive(&sh.tempty[acc]);
+      }
+      // columns [p, p+16) of D0 + D1 of this thread's row
+      auto sum16 = [&](int p, float* sd) {
+        if (parked) {
+          tmem_ld16(ts + (uint32_t)p, sd);
+          tmem_ld_wait();
+        } else {
+          float d1[16];
+          tmem_ld16(t0 + (uint32_t)p, sd);
+          tmem_ld16(t0 + (uint32_t)(rp + p), d1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) sd[e] += d1[e];
+        }
+      };
+      if (!has_work) {
+        // nothing to drain for this warp
+      } else if (I.epi == EPI_FACTOR) {
+        uint16_t* dst = a.work_bf16 + I.dst_off;
+        // one piece: accumulator columns [p, p+16) of this thread's row, old values in `o`
+        auto piece = [&](int p, float (*o)[4]) {
+          float acc16[16];
+          sum16(p, acc16);
           float v[4][4];                 // v[j] = columns 4j .. 4j+3 of this thread's row
 #pragma unroll
           for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) v[j][e] = d0[4 * j + e] + d1[4 * j + e];
+            for (int e = 0; e < 4; ++e) v[j][e] = acc16[4 * j + e];
           // quad transpose, round 1 (partner lane ^ 2): keep the half of the columns this lane's
           // final column group lies in, hand over the other half
           const bool up = (qc & 2) != 0, odd = (qc & 1) != 0;
@@ -394,17 +430,15 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         };
         // the same piece without the turn: this thread's row, columns [p, p+16)
         auto piece_col = [&](int p, float (*o)[4]) {
-          float d0[16], d1[16];
-          tmem_ld16(t0 + (uint32_t)p, d0);
-          tmem_ld16(t0 + (uint32_t)(rp + p), d1);
-          tmem_ld_wait();
+          float sd[16];
+          sum16(p, sd);
           if (own_row >= I.own_count) return;
           float* fp = fbase + own_row + I.k_stride * p;
           uint32_t hi[8], lo[8];
 #pragma unroll
           for (int e = 0; e < 16; e += 2) {
-            const float x0 = p + e < r ? o[e >> 2][e & 3] + I.coef * (d0[e] + d1[e]) : 0.f;
-            const float x1 = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * (d0[e + 1] + d1[e + 1]) : 0.f;
+            const float x0 = p + e < r ? o[e >> 2][e & 3] + I.coef * sd[e] : 0.f;
+            const float x1 = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * sd[e + 1] : 0.f;
             if (p + e < r) __stcg(fp + I.k_stride * e, x0);
             if (p + e + 1 < r) __stcg(fp + I.k_stride * (e + 1), x1);
             split_bf16x2(x0, x1, hi[e >> 1], lo[e >> 1]);
@@ -415,17 +449,15 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
         };
         // and for a row-stored factor with aligned rows
         auto piece_row = [&](int p, float (*o)[4]) {
-          float d0[16], d1[16];
-          tmem_ld16(t0 + (uint32_t)p, d0);
-          tmem_ld16(t0 + (uint32_t)(rp + p), d1);
-          tmem_ld_wait();
+          float sd[16];
+          sum16(p, sd);
           if (own_row >= I.own_count) return;
           float x[16];
           uint32_t hi[8], lo[8];
 #pragma unroll
           for (int e = 0; e < 16; e += 2) {
-            x[e] = p + e < r ? o[e >> 2][e & 3] + I.coef * (d0[e] + d1[e]) : 0.f;
-            x[e + 1] = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * (d0[e + 1] + d1[e + 1]) : 0.f;
+            x[e] = p + e < r ? o[e >> 2][e & 3] + I.coef * sd[e] : 0.f;
+            x[e + 1] = p + e + 1 < r ? o[(e + 1) >> 2][(e + 1) & 3] + I.coef * sd[e + 1] : 0.f;
             split_bf16x2(x[e], x[e + 1], hi[e >> 1], lo[e >> 1]);
           }
           float* fp = fbase + I.own_stride * own_row + p;
@@ -492,8 +524,10 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           }
         }
       }
-      tc_fence_before();
-      mbar_arrive(&sh.tempty[acc]);
+      if (!early) {
+        tc_fence_before();
+        mbar_arrive(&sh.tempty[acc]);
+      }
     }
   }
 
