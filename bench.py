@@ -41,10 +41,9 @@ def _peaks():
             "source": "fallback"}
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload
-# (profiles/ holds the captures these come from).  tc_panel: captured on the 4-layer case gpt2_1p5b@4
-# (446.4 MB per launch) and scaled by 12, since every low-rank block belongs to a layer.
-NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 12 * 492.9e6}
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload, from the
+# single-pass full-size capture summarised in profiles/ (tc_panel: mean of the four launches of a step).
+NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 6.76e9, "tc_apply:gpt2_1p5b:blockmean": 13.13e9}
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
@@ -214,6 +213,12 @@ def kernel_algorithmic_work(kind: str, blocks, gsz: int, k_eff: int):
         fl = sum(4.0 * nb(b) * b.rank + 8.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr) / 4.0
         return "alu", fl, "flops"
     if kind == "tc_panel":
+        # One refit pass.  Measured at full size the launch saturates DRAM (ncu: 6.0 TB/s), so HBM is its bound.
+        # Algorithmic bytes per block: g once; the fp32 factors read and written; the split-bf16 source set and
+        # set 0 read, the next set written: r (m + n) (4 + 4 + 2 * 4 + 4) bytes.
+        tot = sum(nb(b) * gsz + 20 * b.rank * (b.rows + b.cols) for b in lowr)
+        return "hbm", tot, "bytes"
+    if kind == "tc_panel_flops":
         # g R^T and L^T g of one refit pass: 4 m n r per block (hi/lo operand doubling not counted)
         fl = sum(4.0 * nb(b) * b.rank for b in lowr)
         return "tensor", fl, "flops"
@@ -345,10 +350,10 @@ def run_gpu(args) -> None:
     step_bytes = ctx.adapm_step_bytes()
     dom = max(kernels, key=lambda k: kernels[k]["share"]) if kernels else "stream_update"
 
-    def roofline_of(kind):
+    def roofline_of(kind, work=None):
         if kind not in kernels or kernels[kind]["launches_per_step"] == 0:
             return None
-        bound, amount, _ = kernel_algorithmic_work(kind, blocks, gsz, k_eff)
+        bound, amount, _ = kernel_algorithmic_work(work or kind, blocks, gsz, k_eff)
         sec = kernels[kind]["ms_per_step"] / kernels[kind]["launches_per_step"] * 1e-3
         if bound == "hbm":
             ach, peak, unit = amount / sec / 1e9, peaks["hbm_gbs"], "GB/s"
@@ -383,6 +388,8 @@ def run_gpu(args) -> None:
         "kernels": kernels,
         "roofline": roofline_of(dom),
         "roofline_stream_update": roofline_of("stream_update"),
+        "roofline_tc_apply": roofline_of("tc_apply"),
+        "roofline_tc_panel_tensor": roofline_of("tc_panel", "tc_panel_flops"),
         "clocks": clocks,
         "e2e": e2e,
         "cpu_baseline": {"value": 1.0 / cpu_s, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
