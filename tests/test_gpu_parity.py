@@ -245,6 +245,19 @@ def test_tensor_path_can_be_forced_and_refuses_what_it_cannot_address():
     assert e.value.code == -6
 
 
+def test_tensor_path_shallow_rings_partial_tiles_and_every_epilogue_form():
+    """Rank 128 next to a per-element v leaves the apply kernel one g / W buffer and two R stages; the other blocks
+    add a run of 18 column tiles whose last tile is 24 columns wide (quarters past the edge are not stored), five
+    row panels with a ragged last one, and ranks that take the aligned-row, the by-column and the transposing
+    form of the refit epilogue."""
+    blocks = _pack([(300, 384, A.MOM_LOWRANK, 128, A.V_ELEMENT, 0),
+                    (200, 2200, A.MOM_LOWRANK, 24, A.V_BLOCKMEAN, 1),
+                    (520, 136, A.MOM_LOWRANK, 40, A.V_ELEMENT, 0),
+                    (136, 520, A.MOM_LOWRANK, 13, A.V_BLOCKMEAN, 8)])
+    w = WL.Workload("shallow", [], "bf16", "normal", steps=6)
+    _run(w, True, 6, path=A.PATH_TENSOR, blocks=blocks)
+
+
 def test_tensor_path_follows_moving_gradient_buffers():
     """Tensor maps hold absolute addresses; a gradient buffer that moves between steps must be picked up."""
     import torch
