@@ -373,7 +373,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           for (int j = 0; j < 4; ++j)
 #pragma unroll
             for (int e = 0; e < 4; ++e) v[j][e] = acc16[4 * j + e];
-          // quad transpose, round 1 (partner lane ^ 2): keep the half of the columns this lane's
+          // quad transpose, first exchange (partner lane ^ 2): keep the half of the columns this lane's
           // final column group lies in, hand over the other half
           const bool up = (qc & 2) != 0, odd = (qc & 1) != 0;
           float k0[4], k1[4], g0[4], g1[4];
@@ -385,7 +385,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             g0[e] = __shfl_xor_sync(0xffffffffu, s0, 2);
             g1[e] = __shfl_xor_sync(0xffffffffu, s1, 2);
           }
-          // round 2 (partner lane ^ 1): keep this lane's column group of the two rows held so far,
+          // second exchange (partner lane ^ 1): keep this lane's column group of the two rows held so far,
           // hand over the neighbour's; t[0..3] then belong to quad rows qc, qc^2, qc^1, qc^3
           float t[4][4];
 #pragma unroll

@@ -1,6 +1,6 @@
 """GPU-vs-oracle parity through the C ABI: trajectories on the five parameter sets and edge cases.
 
-Tolerances (stated by the benchmark spec): max relative error <= 1e-5 on the fp32 elementwise / reduction paths
+Tolerances: max relative error <= 1e-5 on the fp32 elementwise / reduction paths
 (W, v, m of blocks without or with full momentum; v everywhere) and <= 2e-3 on the contraction paths
 (L, R, P = L R and W of low-rank blocks).  The error of a tensor is max|gpu - ref| / max|ref|.
 """
