@@ -106,6 +106,8 @@ struct TcProgram {
   int final_set = 0;
   // tensor maps: device table + pinned host staging, re-encoded when the buffers move
   CUtensorMap* d_maps = nullptr;
+  int32_t* d_team_counters = nullptr;   // pacing counters of the panel launches (see schedule_panels)
+  int n_teams = 0;
   CUtensorMap* h_maps = nullptr;
   const void* enc_grads = nullptr;
   const void* enc_work = nullptr;
@@ -126,6 +128,7 @@ void destroy_tensor_program(adapm_ctx* c) {
   TcProgram* p = c->tc;
   if (!p) return;
   if (p->d_maps) cudaFree(p->d_maps);
+  if (p->d_team_counters) cudaFree(p->d_team_counters);
   if (p->h_maps) cudaFreeHost(p->h_maps);
   if (p->maps_copied) cudaEventDestroy(p->maps_copied);
   delete p;
@@ -193,6 +196,85 @@ void schedule_items(std::vector<tc::Item>& v, int grid, std::vector<int32_t>& be
     v.insert(v.end(), per[c].begin(), per[c].end());
     begin[c + 1] = (int32_t)v.size();
   }
+}
+
+// The panel items of one block: v[first .. first + n_row) work on row panels (K runs over the columns of g),
+// the next n_col on column panels (K runs over the rows).
+struct BlockSpan {
+  size_t first, n_row, n_col;
+};
+
+// Team schedule for a panel launch.  The row panels and the column panels of a block each read all of g, DRAM is
+// what bounds the launch, and at full size the second read finds nothing in L2 unless it follows the first
+// closely.  So a team of CTAs takes one block at a time: every item of the kind with the longer K loop gets a CTA
+// of its own, the items of the other kind are dealt in order to as many further CTAs as keep pace with them (item
+// j of the short kind covers the j-th slice of the long kind's K range, so both kinds sweep g together), and no
+// CTA of the team starts loading the next block before all have issued the loads of this one (a counter per team
+// that the items wait on and add to; CTAs without work on a block get a filler that only does that).
+// Blocks go to teams longest first.  Returns the number of teams, or 0 after falling back to schedule_items when
+// the blocks are too few to keep teams busy.
+int schedule_panels(std::vector<tc::Item>& v, const std::vector<BlockSpan>& blocks, int grid,
+                    std::vector<int32_t>& begin) {
+  for (auto& it : v) it.cost = item_cost(it);
+  struct Plan { size_t blk; int n_long, n_short_ctas; int64_t duration; bool rows_long; };
+  std::vector<Plan> plans;
+  int team = 1;
+  for (size_t b = 0; b < blocks.size(); ++b) {
+    const BlockSpan& B = blocks[b];
+    if (B.n_row == 0 || B.n_col == 0) { team = grid + 1; break; }
+    const int64_t c_row = v[B.first].cost, c_col = v[B.first + B.n_row].cost;
+    Plan p;
+    p.blk = b; p.rows_long = c_row >= c_col;
+    const int64_t c_long = p.rows_long ? c_row : c_col, c_short = p.rows_long ? c_col : c_row;
+    const size_t n_long = p.rows_long ? B.n_row : B.n_col, n_short = p.rows_long ? B.n_col : B.n_row;
+    p.n_long = (int)n_long;
+    p.n_short_ctas = (int)std::min<int64_t>((int64_t)n_short, ((int64_t)n_short * c_short + c_long - 1) / c_long);
+    p.duration = std::max<int64_t>(c_long, ((int64_t)n_short + p.n_short_ctas - 1) / p.n_short_ctas * c_short);
+    team = std::max(team, p.n_long + p.n_short_ctas);
+    plans.push_back(p);
+  }
+  const int n_teams = team <= grid ? grid / team : 0;
+  if (n_teams == 0 || (int)blocks.size() < 4 * n_teams) {
+    schedule_items(v, grid, begin);
+    return 0;
+  }
+  std::stable_sort(plans.begin(), plans.end(), [](const Plan& a, const Plan& b) { return a.duration > b.duration; });
+  std::vector<std::vector<tc::Item>> per(grid);
+  std::vector<int64_t> load(n_teams, 0);
+  std::vector<int> done(n_teams, 0);      // blocks given to the team so far
+  tc::Item filler;
+  std::memset(&filler, 0, sizeof(filler));
+  filler.epi = tc::EPI_NONE; filler.own1 = -1; filler.rp = 16;
+  for (const Plan& p : plans) {
+    int t = 0;
+    for (int q = 1; q < n_teams; ++q)
+      if (load[q] < load[t]) t = q;
+    load[t] += p.duration;
+    const BlockSpan& B = blocks[p.blk];
+    const size_t long0 = p.rows_long ? B.first : B.first + B.n_row;
+    const size_t short0 = p.rows_long ? B.first + B.n_row : B.first;
+    const size_t n_short = p.rows_long ? B.n_col : B.n_row;
+    const int cta0 = t * team;
+    std::vector<size_t> mark(team);
+    for (int q = 0; q < team; ++q) mark[q] = per[cta0 + q].size();
+    for (int i = 0; i < p.n_long; ++i) per[cta0 + i].push_back(v[long0 + i]);
+    for (size_t j = 0; j < n_short; ++j) per[cta0 + p.n_long + (int)(j % p.n_short_ctas)].push_back(v[short0 + j]);
+    for (int q = 0; q < team; ++q) {
+      std::vector<tc::Item>& mine = per[cta0 + q];
+      if (mine.size() == mark[q]) mine.push_back(filler);
+      for (size_t i = mark[q]; i < mine.size(); ++i) { mine[i].team = (int16_t)t; mine[i].signal = 0; mine[i].wait_count = 0; }
+      mine[mark[q]].wait_count = team * done[t];      // every member has issued the loads of the block before
+      mine.back().signal = 1;
+    }
+    ++done[t];
+  }
+  v.clear();
+  begin.assign(grid + 1, 0);
+  for (int c = 0; c < grid; ++c) {
+    v.insert(v.end(), per[c].begin(), per[c].end());
+    begin[c + 1] = (int32_t)v.size();
+  }
+  return n_teams;
 }
 
 }  // namespace
@@ -278,6 +360,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     const int dst = src == 1 ? 2 : 1;
     const float coef = (float)etas[pass] * a1;
     std::vector<tc::Item> grams, panels;
+    std::vector<BlockSpan> spans;
     for (size_t bi = 0; bi < P->blk.size(); ++bi) {
       const TcBlock& t = P->blk[bi];
       const adapm_block& b = c->blocks[t.id];
@@ -337,17 +420,19 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         panels.push_back(it);
       };
       const int step = pair_panels ? 256 : 128;
+      BlockSpan sp;
+      sp.first = panels.size();
       for (int p0 = 0; p0 < m; p0 += step) panel(true, p0, pair_panels && p0 + 128 < m);
+      sp.n_row = panels.size() - sp.first;
       for (int p0 = 0; p0 < n; p0 += step) panel(false, p0, pair_panels && p0 + 128 < n);
+      sp.n_col = panels.size() - sp.first - sp.n_row;
+      spans.push_back(sp);
     }
-    // (Two schedules that keep a block's row and column panels together in time, so that their two reads of g
-    // could meet in L2 - block order, and teams of CTAs sweeping one block at a time - measured no faster than
-    // longest-first.)
     const int grid_g = (int)std::min<int64_t>((int64_t)grams.size(), P->n_sms);
     const int grid_p = (int)std::min<int64_t>((int64_t)panels.size(), P->n_sms);
     std::vector<int32_t> begin_g, begin_p;
     schedule_items(grams, grid_g, begin_g);
-    schedule_items(panels, grid_p, begin_p);
+    P->n_teams = std::max(P->n_teams, schedule_panels(panels, spans, grid_p, begin_p));
     Launch G{LK_TC_GRAM, append_items(c->h_tables, grams), (int64_t)grams.size(), grid_g};
     G.aux0 = 4 * rp_max; G.aux1 = 8 * rp_max <= 512 ? 2 : 1; G.aux2 = two_a ? 1 : 0;
     G.aux3 = append_items(c->h_tables, begin_g);
@@ -413,6 +498,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
   // ---- tensor maps -------------------------------------------------------------------------------------------------
   const size_t map_bytes = P->blk.size() * kMapsPerBlock * sizeof(CUtensorMap);
   cudaError_t e = cudaMalloc((void**)&P->d_maps, map_bytes);
+  if (e == cudaSuccess && P->n_teams > 0) e = cudaMalloc((void**)&P->d_team_counters, P->n_teams * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMallocHost((void**)&P->h_maps, map_bytes);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&P->maps_copied, cudaEventDisableTiming);
   if (e == cudaSuccess)
@@ -503,6 +589,11 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.stage_bytes = e.stage_bytes; a.n_stages = e.n_stages; a.a_bytes = e.a_bytes;
       a.acc_cols = (int32_t)L.aux0; a.n_acc = (int32_t)L.aux1;
       a.cta_begin = (const int32_t*)(c->d_tables + L.aux3);
+      a.team_counters = nullptr;
+      if (L.kind == LK_TC_PANEL && P->d_team_counters) {
+        ADAPM_CUDA(cudaMemsetAsync(P->d_team_counters, 0, P->n_teams * sizeof(int32_t), s));
+        a.team_counters = P->d_team_counters;
+      }
       // one accumulator buffer of paired panels (4 rp_max columns) leaves room to park their sums (2 rp_max)
       a.sum_col = (L.kind == LK_TC_PANEL && L.aux2 != 0 && a.n_acc == 1 && a.acc_cols + a.acc_cols / 2 <= 512)
                       ? a.acc_cols : -1;

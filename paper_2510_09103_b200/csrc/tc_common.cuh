@@ -24,7 +24,8 @@ constexpr uint32_t kSpinLimit = 1u << 20;          // bounded waits: about a sec
 constexpr uint32_t kSuspendHintNs = 1000;          // a poll may park the thread this long before it reports failure
 
 // status bits a kernel may set when a bounded wait runs out
-enum : int32_t { ST_WAIT_FULL = 1, ST_WAIT_EMPTY = 2, ST_WAIT_TMEM_FULL = 4, ST_WAIT_TMEM_EMPTY = 8, ST_WAIT_DRAIN = 16 };
+enum : int32_t { ST_WAIT_FULL = 1, ST_WAIT_EMPTY = 2, ST_WAIT_TMEM_FULL = 4, ST_WAIT_TMEM_EMPTY = 8, ST_WAIT_DRAIN = 16,
+                 ST_WAIT_TEAM = 32 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

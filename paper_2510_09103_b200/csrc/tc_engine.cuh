@@ -44,7 +44,7 @@ constexpr int kStageK = 128;
 constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 32 KB
 constexpr int kEngineThreads = 320;
 
-enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1 };
+enum : int32_t { EPI_FACTOR = 0, EPI_GRAM = 1, EPI_NONE = 2 };   // EPI_NONE: a filler that only keeps a CTA in step
 
 struct Seg {
   int32_t map_a;             // 2-D tensor map, box 64 x 128
@@ -80,7 +80,11 @@ struct Item {
   int64_t own_stride, k_stride;
   int64_t dst_off;           // bf16 element offset of the destination array in the workspace
   int32_t dst_ld;            // its row pitch in elements
-  int32_t pad_;
+  // Pacing of a team of CTAs that work through the same blocks (so that their reads of g meet in L2): before its
+  // first load the item waits until team_counters[team] >= wait_count, after its last load it adds `signal`.
+  // Pacing only: no data depends on it.
+  int16_t team, signal;
+  int32_t wait_count;
   float coef;
   int32_t cost;              // stages, for scheduling
 };
@@ -106,6 +110,7 @@ struct EngineArgs {
   int32_t n_acc;             // 1 or 2 accumulator buffers
   const int32_t* cta_begin;  // CTA c runs items [cta_begin[c], cta_begin[c + 1]) in order
   int32_t sum_col;           // EPI_FACTOR: first of the tensor-memory columns the epilogue parks D0 + D1 in, or -1
+  int32_t* team_counters;    // one counter per team, zero at launch (nullptr when no item waits)
 };
 
 struct __align__(8) EngineShared {
@@ -148,6 +153,20 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       bool ok = true;
       for (int it = it_begin; it < it_end && ok; ++it) {
         const Item& I = a.items[it];
+        if (I.wait_count > 0) {
+          // bounded like every wait here: a team member that never arrives ends this CTA with a status, not a hang
+          volatile int32_t* cnt = a.team_counters + I.team;
+          uint32_t spin = 0;
+          while (*cnt < I.wait_count) {
+            if (++spin >= kSpinLimit || ((spin & 255u) == 0 && *abort)) { ok = false; break; }
+            __nanosleep(256);
+          }
+          if (!ok) {
+            *abort = 1;
+            atomicOr(a.status, ST_WAIT_TEAM);
+            break;
+          }
+        }
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const Seg S = I.seg[s];
           const CUtensorMap* ma = a.maps + S.map_a;
@@ -173,6 +192,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
           }
         }
+        if (ok && I.signal) atomicAdd(a.team_counters + I.team, (int)I.signal);
       }
       if (!ok) {
         // leave no copy in flight: every stage that was filled must have landed before the CTA exits
