@@ -43,7 +43,7 @@ def _peaks():
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload, from the
 # single-pass full-size capture summarised in profiles/ (tc_panel: mean of the four launches of a step).
-NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 6.76e9, "tc_apply:gpt2_1p5b:blockmean": 13.13e9}
+NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 4.70e9, "tc_apply:gpt2_1p5b:blockmean": 13.18e9}
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
@@ -213,7 +213,7 @@ def kernel_algorithmic_work(kind: str, blocks, gsz: int, k_eff: int):
         fl = sum(4.0 * nb(b) * b.rank + 8.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr) / 4.0
         return "alu", fl, "flops"
     if kind == "tc_panel":
-        # One refit pass.  Measured at full size the launch saturates DRAM (ncu: 6.0 TB/s), so HBM is its bound.
+        # One refit pass.  HBM is the resource it uses most (ncu at full size: 4.7 GB per launch at 4.2 TB/s).
         # Algorithmic bytes per block: g once; the fp32 factors read and written; the split-bf16 source set and
         # set 0 read, the next set written: r (m + n) (4 + 4 + 2 * 4 + 4) bytes.
         tot = sum(nb(b) * gsz + 20 * b.rank * (b.rows + b.cols) for b in lowr)
