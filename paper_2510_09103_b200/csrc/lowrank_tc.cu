@@ -484,10 +484,15 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     P->apply_r_region = l_region;
     P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
     P->apply_buf_bytes = tc::kApplyBufBytes + (any_element_v ? tc::kWBoxBytes : 0);
-    if (226 * 1024 - P->apply_w_region < 2 * P->apply_buf_bytes) {   // two buffers at least: give up R stages
+    auto bufs_with = [&](int r_stages) { return (226 * 1024 - l_region - r_stages * tc::kBoxBytes) / P->apply_buf_bytes; };
+    if (any_element_v && bufs_with(3) < 3 && bufs_with(1) >= 3) {
+      // the larger buffers of a per-element v: a third buffer is worth more than the second and third R stage
+      // (measured on the 1.5B shapes: 9.6 ms with three R stages and two buffers, 8.0 ms with one and three)
+      P->apply_r_stages = 1;
+    } else if (bufs_with(3) < 2) {   // two buffers at least: give up an R stage
       P->apply_r_stages = 2;
-      P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
     }
+    P->apply_w_region = l_region + P->apply_r_stages * tc::kBoxBytes;
     P->apply_bufs = std::max(1, std::min(tc::kApplyMaxBufs, (226 * 1024 - P->apply_w_region) / P->apply_buf_bytes));
     P->smem_apply = P->apply_w_region + P->apply_bufs * P->apply_buf_bytes + 1024;
     Launch A{LK_TC_APPLY, append_items(c->h_tables, items), (int64_t)items.size(),
