@@ -14,6 +14,7 @@
 // rp = rank rounded up to 16; padded columns are kept at zero by every writer.
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 
 #include "adapm_internal.h"
@@ -233,7 +234,11 @@ int schedule_panels(std::vector<tc::Item>& v, const std::vector<BlockSpan>& bloc
     team = std::max(team, p.n_long + p.n_short_ctas);
     plans.push_back(p);
   }
-  const int n_teams = team <= grid ? grid / team : 0;
+  // The pacing assumes that the CTAs of the launch run at the same time (one per SM).  A caller who shares the
+  // GPU with long-running kernels can turn it off: ADAPM_PANEL_TEAMS=0 in the environment at adapm_create.
+  const char* env = std::getenv("ADAPM_PANEL_TEAMS");
+  const bool teams_off = env && env[0] == '0';
+  const int n_teams = (team <= grid && !teams_off) ? grid / team : 0;
   if (n_teams == 0 || (int)blocks.size() < 4 * n_teams) {
     schedule_items(v, grid, begin);
     return 0;

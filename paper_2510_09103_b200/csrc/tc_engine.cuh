@@ -41,6 +41,7 @@ namespace tc {
 
 constexpr int kMaxSegs = 6;
 constexpr int kStageK = 128;
+constexpr uint32_t kTeamSpinLimit = 1u << 24;    // polls of 256 ns each: about four seconds
 constexpr int kStageABytes = 2 * kBoxBytes;      // the A side of a stage: 32 KB
 constexpr int kEngineThreads = 320;
 
@@ -154,11 +155,12 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       for (int it = it_begin; it < it_end && ok; ++it) {
         const Item& I = a.items[it];
         if (I.wait_count > 0) {
-          // bounded like every wait here: a team member that never arrives ends this CTA with a status, not a hang
+          // Bounded like every wait here: a team member that never arrives ends this CTA with a status, not a
+          // hang.  The bound is generous (seconds), because a member may start late when other work holds SMs.
           volatile int32_t* cnt = a.team_counters + I.team;
           uint32_t spin = 0;
           while (*cnt < I.wait_count) {
-            if (++spin >= kSpinLimit || ((spin & 255u) == 0 && *abort)) { ok = false; break; }
+            if (++spin >= kTeamSpinLimit || ((spin & 255u) == 0 && *abort)) { ok = false; break; }
             __nanosleep(256);
           }
           if (!ok) {

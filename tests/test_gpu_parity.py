@@ -295,6 +295,28 @@ def test_tensor_path_is_bitwise_reproducible():
     assert torch.equal(p1, p2) and torch.equal(s1, s2)
 
 
+def test_panel_team_schedule_changes_no_bit(monkeypatch):
+    """The refit's panel launch hands its items to teams of CTAs kept in step by a counter when the set has enough
+    blocks (llama350m has); ADAPM_PANEL_TEAMS=0 hands them out longest-first instead.  Which CTA runs an item, and
+    when, must not change any result."""
+    import torch
+
+    def trajectory(teams):
+        monkeypatch.setenv("ADAPM_PANEL_TEAMS", teams)
+        run = ParityRun(WL.get_workload("llama350m"), True, oracle_blocks=[], lowrank_path=A.PATH_TENSOR)
+        for _ in range(3):
+            run.step()
+        torch.cuda.synchronize()
+        out = run.params.clone(), run.state.clone()
+        assert run.ctx.adapm_get_status() == 0
+        run.close()
+        return out
+
+    p1, s1 = trajectory("1")
+    p0, s0 = trajectory("0")
+    assert torch.equal(p1, p0) and torch.equal(s1, s0)
+
+
 def test_tensor_path_nan_gradient_stays_in_its_block_and_does_not_hang():
     import torch
     blocks = _pack([(256, 128, A.MOM_LOWRANK, 8, A.V_BLOCKMEAN, 1), (128, 128, A.MOM_LOWRANK, 8, A.V_BLOCKMEAN, 1)])
