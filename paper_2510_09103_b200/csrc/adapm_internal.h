@@ -144,7 +144,7 @@ struct Launch {
 // ---------------------------------------------------------------------------------------------
 int launch_stream(const StreamBlk* d_tab, const int32_t* d_cta_blk, int64_t grid, const Bases& b,
                   const StepScalars& sc, int grad_dtype, cudaStream_t s);
-int launch_reduce_partial(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_units, const void* grads,
+int launch_reduce_partial(const ReduceJob* d_tab, const int32_t* d_cta_job, int64_t n_jobs, int64_t n_units, const void* grads,
                           float* work, int grad_dtype, cudaStream_t s);
 int launch_reduce_final(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_groups, float* state, const float* work,
                         float beta2, cudaStream_t s);

@@ -213,7 +213,16 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   auto& prog = c->program;
   if (!rjobs.empty()) {
     const int64_t off = append_table(c->h_tables, rjobs);
-    prog.push_back({LK_REDUCE_PARTIAL, off, (int64_t)rjobs.size(), (unit_cursor + 7) / 8, unit_cursor});
+    // CTA index -> job of the CTA's first unit (the job table is sorted by first_unit), so that a warp finds its job
+    // with a step or two instead of a binary search
+    std::vector<int32_t> cta_job((size_t)((unit_cursor + 7) / 8));
+    for (size_t q = 0, j = 0; q < cta_job.size(); ++q) {
+      while (j + 1 < rjobs.size() && rjobs[j + 1].first_unit <= (int64_t)q * 8) ++j;
+      cta_job[q] = (int32_t)j;
+    }
+    Launch RP{LK_REDUCE_PARTIAL, off, (int64_t)rjobs.size(), (unit_cursor + 7) / 8, unit_cursor};
+    RP.aux1 = append_table(c->h_tables, cta_job);
+    prog.push_back(RP);
     prog.push_back({LK_REDUCE_FINAL, off, (int64_t)rjobs.size(), (group_cursor + 7) / 8, group_cursor});
   }
   if (!sblk.empty()) {
@@ -473,7 +482,9 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
     int rc = ADAPM_OK;
     switch (L.kind) {
       case LK_REDUCE_PARTIAL:
-        rc = launch_reduce_partial((const ReduceJob*)tab, L.n_items, L.aux0, grads, work, hp.grad_dtype, s); break;
+        rc = launch_reduce_partial((const ReduceJob*)tab, (const int32_t*)(c->d_tables + L.aux1), L.n_items, L.aux0, grads,
+                                   work, hp.grad_dtype, s);
+        break;
       case LK_REDUCE_FINAL:
         rc = launch_reduce_final((const ReduceJob*)tab, L.n_items, L.aux0, (float*)state, work, hp.beta2, s); break;
       case LK_STREAM:

@@ -236,17 +236,15 @@ __device__ __forceinline__ float warp_chunk_sumsq(const typename GT::elem* __res
 }
 
 template <typename GT>
-__global__ void __launch_bounds__(256) reduce_partial_kernel(const ReduceJob* __restrict__ tab, int n_jobs,
+__global__ void __launch_bounds__(256) reduce_partial_kernel(const ReduceJob* __restrict__ tab,
+                                                             const int32_t* __restrict__ cta_job, int n_jobs,
                                                              int64_t n_units,
                                                              const typename GT::elem* __restrict__ grads,
                                                              float* __restrict__ work) {
   const int64_t unit = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (unit >= n_units) return;
-  int lo = 0, hi = n_jobs - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (tab[mid].first_unit <= unit) lo = mid; else hi = mid - 1;
-  }
+  int lo = cta_job[blockIdx.x];                       // job of the CTA's first unit; this warp's is at most 7 units on
+  while (lo + 1 < n_jobs && tab[lo + 1].first_unit <= unit) ++lo;
   const ReduceJob J = tab[lo];
   const int64_t u = unit - J.first_unit;
   const int64_t group = u / J.chunks_per_group;
@@ -344,14 +342,15 @@ int launch_stream(const StreamBlk* d_tab, const int32_t* d_cta_blk, int64_t grid
   return ADAPM_OK;
 }
 
-int launch_reduce_partial(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_units, const void* grads, float* work,
-                          int grad_dtype, cudaStream_t s) {
+int launch_reduce_partial(const ReduceJob* d_tab, const int32_t* d_cta_job, int64_t n_jobs, int64_t n_units,
+                          const void* grads, float* work, int grad_dtype, cudaStream_t s) {
   if (n_units <= 0) return ADAPM_OK;
   const unsigned grid = (unsigned)((n_units + 7) / 8);
   if (grad_dtype == ADAPM_GRAD_BF16)
-    reduce_partial_kernel<GradBF16><<<grid, 256, 0, s>>>(d_tab, (int)n_jobs, n_units, (const uint16_t*)grads, work);
+    reduce_partial_kernel<GradBF16><<<grid, 256, 0, s>>>(d_tab, d_cta_job, (int)n_jobs, n_units, (const uint16_t*)grads,
+                                                         work);
   else
-    reduce_partial_kernel<GradF32><<<grid, 256, 0, s>>>(d_tab, (int)n_jobs, n_units, (const float*)grads, work);
+    reduce_partial_kernel<GradF32><<<grid, 256, 0, s>>>(d_tab, d_cta_job, (int)n_jobs, n_units, (const float*)grads, work);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }
