@@ -26,6 +26,13 @@ Readings of the paper taken here (each is a choice; the paper does not settle it
     hence m_1 is unchanged) and L_0 is given orthonormal columns: Gaussian draws
     orthonormalised by modified Gram-Schmidt, rounded to fp32 (`init_L0`).
   * "No momentum" blocks use m^c_t = g_t.
+  * "Global gradient clipping at a threshold of 1.0" (Section 5.1, Setups) is the usual clipping by the global
+    norm: with n = the 2-norm of all gradients of the step taken together, every gradient is multiplied by
+    s = min(1, c / n) before Algorithm 1 sees it (lines 4 and 7 both use the clipped gradient).  n = 0 gives s = 1.
+  * The ablation "without bias correction" (Section 5.1.2, Fig. 4a) is read as m^c := m_t, i.e. Eq. 3 left out
+    and nothing else changed.  Section 4.2's phrase "directly applying L_t R_t as the momentum" would instead
+    give m^c := L_t R_t; the two differ by the residual r_t.  `correction=False` takes the first reading and
+    `correction_off_uses_product=True` the second.
 Parity with the authors' unreleased code on these readings is unpinned; what is
 pinned (tests/test_oracle_pins.py) is this oracle against closed forms, special
 cases, a library optimizer, the proof identity of Theorem 2 and brute force.
@@ -75,6 +82,8 @@ class HParams:
     inner_lr_scale: float = 1.0  # multiplies every eta_k; 1 = as printed
     adam_debias: bool = False
     correction: bool = True      # Eq. 3 on; off: m^c := m_t
+    correction_off_uses_product: bool = False   # with correction off: m^c := L_t R_t instead of m_t
+    max_grad_norm: float = math.inf   # global clipping threshold c; inf disables
 
 
 @dataclass
@@ -169,11 +178,28 @@ def new_state(blk: Block, L0: Optional[np.ndarray] = None) -> BlockState:
     return st
 
 
+def global_clip_scale(grads, max_grad_norm: float) -> float:
+    """s = min(1, c / ||g||_2) with the norm taken over all gradients of the step (Section 5.1, Setups)."""
+    if not math.isfinite(max_grad_norm):
+        return 1.0
+    total = 0.0
+    for g in grads:
+        g = np.asarray(g, dtype=np.float64)
+        total += float(np.sum(g * g))
+    norm = math.sqrt(total)
+    if norm == 0.0:
+        return 1.0
+    return min(1.0, max_grad_norm / norm)
+
+
 def block_step(W: np.ndarray, g: np.ndarray, st: BlockState, blk: Block, hp: HParams, t: int,
-               solver: str = "gd", keep: bool = False) -> np.ndarray:
-    """Advance one block by one step (t is 1-based).  Returns W_{t+1}; updates `st` in place."""
+               solver: str = "gd", keep: bool = False, gscale: float = 1.0) -> np.ndarray:
+    """Advance one block by one step (t is 1-based).  Returns W_{t+1}; updates `st` in place.
+    `gscale` is the step's global clipping factor (global_clip_scale over ALL blocks' gradients)."""
     W = np.asarray(W, dtype=np.float64).reshape(blk.rows, blk.cols)
     g = np.asarray(g, dtype=np.float64).reshape(blk.rows, blk.cols)
+    if gscale != 1.0:
+        g = gscale * g
     b1 = hp.beta1
 
     # line 7 (or its group average)
@@ -194,7 +220,10 @@ def block_step(W: np.ndarray, g: np.ndarray, st: BlockState, blk: Block, hp: HPa
         else:
             raise ValueError(solver)
         r_t = L @ R - m_t                                       # line 6
-        m_c = m_t - (b1 * r_t) / (1.0 - b1) if hp.correction else m_t   # line 8
+        if hp.correction:
+            m_c = m_t - (b1 * r_t) / (1.0 - b1)                # line 8
+        else:
+            m_c = L @ R if hp.correction_off_uses_product else m_t
         st.L, st.R = L, R
         if keep:
             st.last = {"m_t": m_t, "r_t": r_t, "P_prev": P_prev, "P": L @ R}
@@ -239,7 +268,8 @@ class AdaPMOracle:
     def step(self, params: List[np.ndarray], grads: List[np.ndarray], solver: str = "gd",
              keep: bool = False) -> List[np.ndarray]:
         self.t += 1
-        return [block_step(W, g, st, b, self.hp, self.t, solver, keep)
+        s = global_clip_scale(grads, self.hp.max_grad_norm)
+        return [block_step(W, g, st, b, self.hp, self.t, solver, keep, gscale=s)
                 for W, g, st, b in zip(params, grads, self.states, self.blocks)]
 
     def state_floats(self) -> int:

@@ -378,3 +378,139 @@ def test_weight_decay_is_decoupled_and_clip_is_elementwise():
     hp2 = O.HParams(lr=1.0, beta2=1.0, eps=0.0)
     W2 = O.block_step(np.zeros((1, 2)), np.array([[10.0, 0.25]]), st2, blk2, hp2, 1)
     np.testing.assert_allclose(W2, [[-1.0, -0.25]], rtol=1e-15)
+
+
+# ------------------------------------------------------------------------------------ global gradient-norm clipping
+
+def _three_blocks():
+    blks = [O.Block(6, 5, O.MOM_FULL, weight_decay=0.1), O.Block(4, 7, O.MOM_NONE, lr_scale=0.75, weight_decay=0.1),
+            O.Block(8, 6, O.MOM_LOWRANK, rank=2, v_mode=O.V_BLOCKMEAN, v_group_rows=2, weight_decay=0.1)]
+    return blks
+
+
+def test_clip_below_threshold_changes_nothing():
+    """||g|| <= c gives s = 1: the clipped optimizer is the unclipped one, bit for bit."""
+    blks = _three_blocks()
+    a = O.AdaPMOracle(blks, O.HParams(max_grad_norm=1.0))
+    b = O.AdaPMOracle(blks, O.HParams())
+    Wa = [RNG.standard_normal((k.rows, k.cols)) for k in blks]
+    Wb = [w.copy() for w in Wa]
+    for _ in range(5):
+        g = [RNG.standard_normal((k.rows, k.cols)) * 1e-3 for k in blks]      # norm ~ 0.01
+        assert O.global_clip_scale(g, 1.0) == 1.0
+        Wa, Wb = a.step(Wa, g), b.step(Wb, g)
+        for x, y in zip(Wa, Wb):
+            assert np.array_equal(x, y)
+
+
+def test_clip_scale_is_threshold_over_global_norm():
+    """Hand numbers: gradients (3, 4) and (12,) have global norm 13; c = 1 gives s = 1/13, c = 26 gives 1."""
+    g = [np.array([[3.0, 4.0]]), np.array([[12.0]])]
+    assert O.global_clip_scale(g, 1.0) == pytest.approx(1.0 / 13.0, rel=1e-15)
+    assert O.global_clip_scale(g, 26.0) == 1.0
+    assert O.global_clip_scale(g, math.inf) == 1.0
+    assert O.global_clip_scale([np.zeros((2, 2))], 1.0) == 1.0
+    # the norm is over all blocks together, not per block
+    assert O.global_clip_scale(g[:1], 1.0) == pytest.approx(1.0 / 5.0, rel=1e-15)
+
+
+def test_clip_constant_gradient_closed_forms_use_the_scaled_gradient():
+    """P3 with clipping: a constant gradient g of global norm n > c behaves like the constant gradient (c/n) g."""
+    b1, b2, c = 0.9, 0.95, 0.5
+    blk = O.Block(4, 6, O.MOM_FULL)
+    g = RNG.standard_normal((4, 6))
+    s = c / np.linalg.norm(g)
+    orc = O.AdaPMOracle([blk], O.HParams(max_grad_norm=c, clip=math.inf, beta1=b1, beta2=b2))
+    W = [np.zeros((4, 6))]
+    for t in range(1, 9):
+        W = orc.step(W, [g])
+        np.testing.assert_allclose(orc.states[0].m, (1 - b1 ** t) * s * g, rtol=1e-13)
+        np.testing.assert_allclose(orc.states[0].v, (1 - b2 ** t) * (s * g) ** 2, rtol=1e-13)
+
+
+def test_clip_matches_torch_clip_grad_norm_then_adamw():
+    """All blocks FULL, debiased, no elementwise clamp: torch.nn.utils.clip_grad_norm_ followed by
+    torch.optim.AdamW.  (torch divides by norm + 1e-6, hence the 2e-6 relative tolerance.)"""
+    torch = pytest.importorskip("torch")
+    shapes = [(5, 4), (3, 7), (1, 6)]
+    W0 = [RNG.standard_normal(sh) for sh in shapes]
+    ps = [torch.nn.Parameter(torch.tensor(w, dtype=torch.float64)) for w in W0]
+    opt = torch.optim.AdamW(ps, lr=2e-3, betas=(0.9, 0.95), eps=1e-8, weight_decay=0.1)
+    blks = [O.Block(r, c, O.MOM_FULL, weight_decay=0.1) for r, c in shapes]
+    orc = O.AdaPMOracle(blks, O.HParams(lr=2e-3, clip=math.inf, adam_debias=True, max_grad_norm=1.0))
+    W = [w.copy() for w in W0]
+    for t in range(1, 9):
+        g = [RNG.standard_normal(sh) * (3.0 if t % 2 else 0.05) for sh in shapes]     # above and below the threshold
+        for p, gi in zip(ps, g):
+            p.grad = torch.tensor(gi, dtype=torch.float64)
+        torch.nn.utils.clip_grad_norm_(ps, 1.0)
+        opt.step()
+        W = orc.step(W, g)
+        for w, p in zip(W, ps):
+            np.testing.assert_allclose(w, p.detach().numpy(), rtol=2e-6, atol=1e-9)
+
+
+def test_clip_applies_before_the_lowrank_target_and_the_second_moment():
+    """The low-rank block sees s g in line 4 and in line 7: feeding the oracle s g without clipping is the same."""
+    blk = O.Block(8, 6, O.MOM_LOWRANK, rank=2, v_mode=O.V_BLOCKMEAN, v_group_rows=2, weight_decay=0.1)
+    L0 = O.init_L0(8, 2, 0, 0)
+    a, b = O.new_state(blk, L0), O.new_state(blk, L0)
+    hp = O.HParams()
+    Wa = RNG.standard_normal((8, 6)); Wb = Wa.copy()
+    for t in range(1, 6):
+        g = RNG.standard_normal((8, 6))
+        s = O.global_clip_scale([g], 0.3)
+        assert s < 1.0
+        Wa = O.block_step(Wa, g, a, blk, hp, t, gscale=s)
+        Wb = O.block_step(Wb, s * g, b, blk, hp, t)
+        assert np.array_equal(Wa, Wb) and np.array_equal(a.L, b.L) and np.array_equal(a.v, b.v)
+
+
+# ------------------------------------------------------------------------------------ ablation switches
+
+def test_correction_off_is_the_uncorrected_target_and_the_product_reading_differs_by_the_residual():
+    """With Eq. 3 left out the update uses m_t (line 4) as it stands; the other reading of Section 4.2 uses L_t R_t.
+    Their difference is the residual r_t of line 6, and with the correction on m^c = m_t - c r_t."""
+    blk = O.Block(6, 5, O.MOM_LOWRANK, rank=2)
+    L0 = O.init_L0(6, 2, 0, 0)
+    W = RNG.standard_normal((6, 5))
+    g = RNG.standard_normal((6, 5)) * 1e-2
+    outs = {}
+    for name, hp in (("on", O.HParams()), ("off", O.HParams(correction=False)),
+                     ("product", O.HParams(correction=False, correction_off_uses_product=True))):
+        st = O.new_state(blk, L0)
+        st.R = RNG.standard_normal((2, 5)) * 1e-2          # a non-trivial previous product
+        RNG2 = np.random.default_rng(3)
+        st.R = RNG2.standard_normal((2, 5)) * 1e-2
+        O.block_step(W, g, st, blk, hp, 1, keep=True)
+        outs[name] = st.last
+    m_t, r_t = outs["on"]["m_t"], outs["on"]["r_t"]
+    b1 = 0.9
+    np.testing.assert_allclose(outs["off"]["m_c"], m_t, rtol=0, atol=0)
+    np.testing.assert_allclose(outs["product"]["m_c"] - outs["off"]["m_c"], r_t, rtol=1e-12, atol=1e-18)
+    np.testing.assert_allclose(outs["on"]["m_c"], m_t - b1 / (1 - b1) * r_t, rtol=1e-12, atol=1e-18)
+    # and the uncorrected target itself, from its definition
+    P_prev = L0 @ (np.random.default_rng(3).standard_normal((2, 5)) * 1e-2)
+    np.testing.assert_allclose(m_t, (1 - b1) * g + b1 * P_prev, rtol=1e-13)
+
+
+def test_inner_lr_scale_multiplies_every_step_size():
+    """inner_lr_scale = s runs Algorithm 2 with s eta_k: the same as the scalar loops of the brute-force pin with
+    the schedule scaled, and s = 0 leaves the factors where they were."""
+    m, n = 3, 2
+    tgt = RNG.standard_normal((m, n))
+    L0 = RNG.standard_normal((m, 1)); R0 = RNG.standard_normal((1, n))
+    s = 0.37
+    L, R = O.lowrank_refit_gd(tgt, L0, R0, 5, s)
+    l = [float(x) for x in L0[:, 0]]; r = [float(x) for x in R0[0]]
+    for k in range(1, 6):
+        eta = s * 0.5 * (1.0 + math.cos(math.pi * k / 5))
+        e = [[l[i] * r[j] - tgt[i, j] for j in range(n)] for i in range(m)]
+        dl = [sum(e[i][j] * r[j] for j in range(n)) for i in range(m)]
+        dr = [sum(l[i] * e[i][j] for i in range(m)) for j in range(n)]
+        l = [l[i] - eta * dl[i] for i in range(m)]
+        r = [r[j] - eta * dr[j] for j in range(n)]
+    np.testing.assert_allclose(L[:, 0], l, rtol=1e-13)
+    np.testing.assert_allclose(R[0], r, rtol=1e-13)
+    L2, R2 = O.lowrank_refit_gd(tgt, L0, R0, 5, 0.0)
+    assert np.array_equal(L2, L0) and np.array_equal(R2, R0)
