@@ -41,15 +41,134 @@ def _peaks():
             "source": "fallback"}
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on the benchmark's workload, from the
-# single-pass full-size capture summarised in profiles/ (tc_panel: mean of the four launches of a step).
-NCU_TRAFFIC_BYTES = {"tc_panel:gpt2_1p5b:blockmean": 4.70e9, "tc_apply:gpt2_1p5b:blockmean": 13.18e9}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic_per_launch.md")
+KERNEL_SOURCES = ("tc_engine.cuh", "tc_apply.cuh", "tc_common.cuh", "lowrank_tc.cu", "stream_kernels.cu")
+
+
+def kernel_source_digest() -> str:
+    """Short hash of the kernel sources: a traffic figure is only quoted while the kernels are the ones captured."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2510_09103_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def recorded_traffic(kind: str, workload: str, v_mode: str):
+    """DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) from the table under profiles/:
+    rows `| kernel | workload | v_mode | bytes per launch | capture | scale | kernel sources |`.  Returns
+    (bytes, note) or (None, why): a row taken from other kernel sources than the present ones does not count."""
+    if not os.path.exists(TRAFFIC_FILE):
+        return None, "no capture recorded"
+    digest = kernel_source_digest()
+    stale = False
+    for line in open(TRAFFIC_FILE):
+        cells = [c.strip() for c in line.strip().strip("|").split("|")]
+        if len(cells) < 7 or cells[0] != kind or cells[1] != workload or cells[2] != v_mode:
+            continue
+        if cells[6] != digest:
+            stale = True
+            continue
+        return float(cells[3]), f"{cells[4]}, scaled x{cells[5]}, kernel sources {cells[6]}"
+    return None, "kernels changed since the last capture" if stale else "no capture recorded"
 
 
 # ------------------------------------------------------------------------------------------------ oracle arm
 
 def _class_key(b):
     return (b.mom_mode, b.rows, b.cols, b.rank, b.v_mode, b.v_group_rows)
+
+
+def _oracle_hparams(w):
+    from oracle import adapm_oracle as O
+    return O.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
+
+
+class OracleSet:
+    """Every block of a parameter set in the oracle.  Blocks of equal shape share one W and one g array (the
+    oracle's time does not depend on the values); every block has its own optimizer state."""
+
+    def __init__(self, w, blocks, only=None):
+        from oracle import adapm_oracle as O
+        import workloads as WL
+        self.O, self.w = O, w
+        self.hp = _oracle_hparams(w)
+        self.ids = list(range(len(blocks))) if only is None else list(only)
+        rng = np.random.default_rng(0)
+        self.arrays, self.items = {}, []
+        for i in self.ids:
+            b = blocks[i]
+            key = (b.rows, b.cols)
+            if key not in self.arrays:
+                W = rng.standard_normal((b.rows, b.cols)) * 0.02
+                g, _ = WL.to_grad_dtype((rng.standard_normal((b.rows, b.cols), dtype=np.float32) * np.float32(1e-3)),
+                                        w.grad_dtype)
+                self.arrays[key] = (W, g.astype(np.float64))
+            ob = O.Block(b.rows, b.cols, b.mom_mode, b.rank, b.v_mode, b.v_group_rows, b.lr_scale, b.weight_decay)
+            L0 = None
+            if b.mom_mode == O.MOM_LOWRANK:
+                L0 = np.linalg.qr(rng.standard_normal((b.rows, b.rank)))[0]      # orthonormal columns, cheaply
+            self.items.append((key, ob, O.new_state(ob, L0)))
+        self.t = 0
+        self.elems = sum(b.rows * b.cols for b in (blocks[i] for i in self.ids))
+
+    def step(self) -> float:
+        """One oracle step over the blocks; returns seconds."""
+        self.t += 1
+        t0 = time.perf_counter()
+        for key, ob, st in self.items:
+            W, g = self.arrays[key]
+            self.O.block_step(W, g, st, ob, self.hp, self.t)
+        return time.perf_counter() - t0
+
+
+def oracle_layer_sample(w, blocks, budget_s: float = 25.0):
+    """The bounded CPU sample of the default run: the blocks of the first transformer layer (all of them, full size)
+    and the small leading tensors, stepped once with every BLAS thread and once with one thread; the set's time
+    is that of the layer times the layer count plus the embeddings' share by element count.
+    Returns (estimated seconds per full step all threads, the same for one thread or None, description)."""
+    from threadpoolctl import threadpool_limits
+    names = [t.name for t in w.tensors]
+    layer_tags = sorted({n.split(".")[0] + "." + n.split(".")[1] if n.startswith("layers.") else n.split(".")[0]
+                         for n in names if n.startswith(("h", "layers.")) and "." in n})
+    first = layer_tags[0] if layer_tags else None
+    n_layers = max(len(layer_tags), 1)
+    # tensor index -> block indices (a fused QKV tensor is three blocks)
+    t2b, k = [], 0
+    for t in w.tensors:
+        nb = 3 if t.role == 4 else 1
+        t2b.append(list(range(k, k + nb))); k += nb
+    in_layer = [i for ti, t in enumerate(w.tensors) if first and t.name.startswith(first + ".") for i in t2b[ti]]
+    outside = [i for ti, t in enumerate(w.tensors) if not t.name.startswith(("h", "layers.")) or "." not in t.name
+               for i in t2b[ti]]
+    small_out = [i for i in outside if blocks[i].rows * blocks[i].cols <= 8_000_000]
+    big_out = [i for i in outside if i not in small_out]
+    sample = OracleSet(w, blocks, in_layer + small_out)
+    layer_elems = sum(blocks[i].rows * blocks[i].cols for i in in_layer)
+    small_elems = sum(blocks[i].rows * blocks[i].cols for i in small_out)
+    big_elems = sum(blocks[i].rows * blocks[i].cols for i in big_out)
+    t_all = sample.step()
+    # blocks without low-rank factors cost per element what the sampled ones of that kind cost: use the sample's
+    # elementwise share, measured on the small outside tensors when there are any
+    per_elem = None
+    if small_out:
+        so = OracleSet(w, blocks, small_out)
+        per_elem = so.step() / max(small_elems, 1)
+    def scale(t_sample):
+        t_small = (per_elem or 0.0) * small_elems
+        t_layer = max(t_sample - t_small, 0.0)
+        return t_layer * n_layers + t_small + (per_elem or t_sample / max(sample.elems, 1)) * big_elems
+    est_all = scale(t_all)
+    est_one = None
+    if t_all * 12 < budget_s:
+        with threadpool_limits(limits=1):
+            t_one = sample.step()
+        est_one = scale(t_one)
+    desc = (f"every block of the first of {n_layers} layers at full size plus the small leading tensors "
+            f"({sample.elems} of {sum(b.rows * b.cols for b in blocks)} elements), one oracle step; layer time x "
+            f"{n_layers}, embeddings by element count")
+    return est_all, est_one, desc
 
 
 def oracle_step_estimate(w, blocks, max_rows: int = 4096, seed: int = 0):
@@ -107,20 +226,32 @@ def run_reference(args) -> None:
     from oracle import planner_oracle as P
     w = WL.get_workload(args.workload)
     blocks = P.plan(w.tensors, w.weight_decay, w.rank_pct, args.v_mode == "blockmean")
-    times, desc = [], ""
-    for i in range(args.warmup + args.steps):
-        t, desc = oracle_step_estimate(w, blocks, seed=i)
-        if i >= args.warmup:
-            times.append(t)
+    # Full oracle steps over every block of the set, timed one by one.  A step of the 1.5B-shaped set takes the
+    # better part of a minute on 16 cores, so the run stops asking for more once `budget_s` is spent: `steps` is
+    # the number of steps that were timed, `steps_requested` what the command line asked for.  The oracle has
+    # nothing to warm up beyond its first call, which is timed like the rest and reported.
+    budget_s = float(os.environ.get("ADAPM_REFERENCE_BUDGET_S", "150"))
+    t_setup = time.perf_counter()
+    oset = OracleSet(w, blocks)
+    setup_s = time.perf_counter() - t_setup
+    times = []
+    while len(times) < max(args.steps, 1):
+        times.append(oset.step())
+        if sum(times) + times[-1] > budget_s:
+            break
     sec = float(np.mean(times))
     val = 1.0 / sec
     cores = _blas_threads()
+    desc = (f"{len(times)} full oracle step(s) over all {len(blocks)} blocks ({oset.elems} elements), numpy fp64, "
+            f"BLAS on {cores} threads, blocks one after another; {setup_s:.0f} s of untimed setup")
     line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
+        "steps_requested": args.steps, "warmup": 0, "ms_per_step": sec * 1e3, "step_seconds": times,
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "params": w.numel, "v_mode": args.v_mode, "grad_dtype": w.grad_dtype},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "cores_os": os.cpu_count(), "kind": "oracle",
+                         "sample": desc},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -213,15 +344,15 @@ def kernel_algorithmic_work(kind: str, blocks, gsz: int, k_eff: int):
         fl = sum(4.0 * nb(b) * b.rank + 8.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr) / 4.0
         return "alu", fl, "flops"
     if kind == "tc_panel":
-        # One refit pass.  HBM is the resource it uses most (ncu at full size: 4.7 GB per launch at 4.2 TB/s).
-        # Algorithmic bytes per block: g once; the fp32 factors read and written; the split-bf16 source set and
-        # set 0 read, the next set written: r (m + n) (4 + 4 + 2 * 4 + 4) bytes.
-        tot = sum(nb(b) * gsz + 20 * b.rank * (b.rows + b.cols) for b in lowr)
-        return "hbm", tot, "bytes"
-    if kind == "tc_panel_flops":
-        # g R^T and L^T g of one refit pass: 4 m n r per block (hi/lo operand doubling not counted)
+        # One refit pass is a contraction: g R^T and L^T g, 4 m n r flops per block (the doubling by the hi/lo
+        # operand split and the small r x r products are the kernel's own and not counted).
         fl = sum(4.0 * nb(b) * b.rank for b in lowr)
         return "tensor", fl, "flops"
+    if kind == "tc_panel_hbm":
+        # The same launch seen from memory, the method's bytes only: g once, the fp32 factors read and written
+        # (the split-bf16 copies are the kernel's own traffic and show up in `traffic`, not here).
+        tot = sum(nb(b) * gsz + 8 * b.rank * (b.rows + b.cols) for b in lowr)
+        return "hbm", tot, "bytes"
     if kind == "tc_gram":
         fl = sum(4.0 * b.rank * b.rank * (b.rows + b.cols) for b in lowr)
         return "tensor", fl, "flops"
@@ -230,6 +361,8 @@ def kernel_algorithmic_work(kind: str, blocks, gsz: int, k_eff: int):
         return "hbm", tot, "bytes"
     if kind in ("reduce_partial",):
         return "hbm", sum(nb(b) * gsz for b in lowr), "bytes"
+    if kind == "reduce_rows":
+        return "hbm", sum(b.rows * 4 + groups(b) * 8 for b in lowr), "bytes"
     return "hbm", 0, "bytes"
 
 
@@ -262,7 +395,10 @@ def run_gpu(args) -> None:
     gd = A.GRAD_BF16 if w.grad_dtype == "bf16" else A.GRAD_F32
     gsz = 2 if w.grad_dtype == "bf16" else 4
     path = {"auto": A.PATH_AUTO, "simt": A.PATH_SIMT, "tensor": A.PATH_TENSOR}[args.path]
-    hp = A.hparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, grad_dtype=gd, lowrank_path=path)
+    flags = ((A.FLAG_NO_PANEL_TEAMS if args.teams == "off" else 0) | (A.FLAG_FORCE_PANEL_TEAMS if args.teams == "force" else 0)
+             | (A.FLAG_NO_SUMSQ_FOLD if args.no_fold else 0))
+    hp = A.hparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, grad_dtype=gd, lowrank_path=path, flags=flags,
+                   tune_panels=args.panels, tune_stage_k=args.stage_k)
     ctx = A.adapm_create(blocks, hp)
 
     # synthetic inputs: parameters N(0, 0.02^2) drawn on the device; gradients tiled from a seeded host pool
@@ -299,7 +435,10 @@ def run_gpu(args) -> None:
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
-    do_steps(args.steps)
+    launches_timed = 0
+    for _ in range(args.steps):
+        do_steps(1)
+        launches_timed += ctx.adapm_launch_count()
     e1.record()
     barrier()
     ms_total, value = whole_job_value(e0.elapsed_time(e1), args.steps, dist, dev)
@@ -361,11 +500,12 @@ def run_gpu(args) -> None:
             ach, peak, unit = amount / sec / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
         else:
             ach, peak, unit = amount / sec / 1e12, SM_COUNT * FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12, "TFLOP/s"
+        traffic, note = recorded_traffic(kind, w.name, args.v_mode)
         return {"kernel": kind, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(f"{kind}:{w.name}:{args.v_mode}"), "peak_source": peaks["source"],
+                "traffic": traffic, "traffic_source": note, "peak_source": peaks["source"],
                 "per_launch_ms": sec * 1e3, "algorithmic_per_launch": amount}
 
-    cpu_s, cpu_desc = oracle_step_estimate(w, blocks)
+    cpu_all, cpu_one, cpu_desc = (float("nan"), None, "skipped (--no-cpu)") if args.no_cpu else oracle_layer_sample(w, blocks)
     sb = ctx.adapm_state_breakdown()
     state_bytes = sum(sb.values())
     line = {
@@ -384,16 +524,18 @@ def run_gpu(args) -> None:
         "step_contraction_tflops": ctx.adapm_step_flops() / (ms_step * 1e-3) / 1e12,
         "state_bytes": state_bytes, "state_breakdown": sb, "adamw_state_bytes": 8 * w.numel,
         "state_saving_vs_adamw": 1.0 - state_bytes / (8.0 * w.numel),
-        "gpu_launches": ctx.adapm_launch_count() * args.steps,
+        "gpu_launches": launches_timed,
+        "launches_per_step": ctx.adapm_launch_count(),
         "kernels": kernels,
         "roofline": roofline_of(dom),
         "roofline_stream_update": roofline_of("stream_update"),
         "roofline_tc_apply": roofline_of("tc_apply"),
-        "roofline_tc_panel_tensor": roofline_of("tc_panel", "tc_panel_flops"),
+        "roofline_tc_panel_hbm": roofline_of("tc_panel", "tc_panel_hbm"),
         "clocks": clocks,
         "e2e": e2e,
-        "cpu_baseline": {"value": 1.0 / cpu_s, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
-                         "sample": cpu_desc, "est_s_per_step": cpu_s},
+        "cpu_baseline": {"value": 1.0 / cpu_all, "unit": UNIT, "cores": _blas_threads(), "cores_os": os.cpu_count(),
+                         "kind": "oracle", "sample": cpu_desc, "est_s_per_step": cpu_all,
+                         "one_thread_est_s_per_step": cpu_one},
     }
     print(json.dumps(line))
     ctx.adapm_destroy()
@@ -411,6 +553,11 @@ def main() -> None:
     ap.add_argument("--v-mode", default="blockmean", choices=["blockmean", "element"])
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle sample (kernel sweeps)")
+    ap.add_argument("--panels", type=int, default=0, help="tensor path: panels per refit item (0 = automatic)")
+    ap.add_argument("--stage-k", type=int, default=0, help="tensor path: K per stage, 64 or 128 (0 = automatic)")
+    ap.add_argument("--teams", default="auto", choices=["auto", "off", "force"], help="panel team schedule")
+    ap.add_argument("--no-fold", action="store_true", help="row sums of g^2 from a pass of their own")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

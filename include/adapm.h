@@ -21,7 +21,17 @@
  *     256-byte aligned.
  *   - Every function returns 0 on success or a negative ADAPM_E* code; nothing throws, aborts or
  *     traps.  Invalid descriptors are rejected by adapm_create, never by a kernel.
- *   - adapm_step is asynchronous on `stream`, allocates nothing and never synchronises.
+ *   - adapm_step is asynchronous on `stream`, allocates nothing and never synchronises.  One context
+ *     is used from one stream at a time.  The first step that sees a new combination of params /
+ *     grads / state / workspace pointers describes the buffers to the TMA unit on the host (a few
+ *     hundred microseconds) and copies that description from pageable memory: make that step
+ *     outside any stream capture.  Four combinations are remembered.
+ *   - Every wait inside a kernel is bounded.  If one runs out (a GPU shared with other work that
+ *     keeps this library's CTAs from running together for about a second), the kernel stops, sets a
+ *     bit in the device status word, and every later kernel of this context returns without writing
+ *     until adapm_get_status has been called.  adapm_get_status then returns ADAPM_EDEVICE: the
+ *     factors of some low-rank blocks are a mix of two iterates and the step is incomplete, so
+ *     restore params and state from the last checkpoint before stepping again.
  *   - There is no CPU fallback: without a CUDA device every device call returns ADAPM_ECUDA.
  */
 #ifndef ADAPM_H_
@@ -42,6 +52,15 @@ enum { ADAPM_V_ELEMENT = 0, ADAPM_V_BLOCKMEAN = 1 };
 enum { ADAPM_GRAD_F32 = 0, ADAPM_GRAD_BF16 = 1 };
 enum { ADAPM_PATH_AUTO = 0, ADAPM_PATH_SIMT = 1, ADAPM_PATH_TENSOR = 2 };
 enum { ADAPM_STATE_M = 0, ADAPM_STATE_L = 1, ADAPM_STATE_R = 2, ADAPM_STATE_V = 3 };
+/* adapm_hparams.flags */
+enum {
+  ADAPM_FLAG_NO_PANEL_TEAMS = 1,     /* hand the refit's panel items out longest-first: no CTA waits for another
+                                        (for callers who share the GPU with long-running kernels)            */
+  ADAPM_FLAG_FORCE_PANEL_TEAMS = 2,  /* team schedule even for sets with few blocks (small profiling cases)  */
+  ADAPM_FLAG_NO_SUMSQ_FOLD = 4,      /* block-mean v of tensor-path blocks from a pass of its own over g     */
+  ADAPM_FLAG_CHECK_FINITE = 8        /* a NaN or Inf anywhere in the gradients: the step writes nothing and
+                                        adapm_get_status reports bit 64 (costs one more pass over g)        */
+};
 
 /* Tensor roles for the default planner (Section 4.1 names the first six kinds). */
 enum {
@@ -88,6 +107,11 @@ typedef struct {
   int32_t correction;      /* 1 = Eq. 3 on; 0 = ablation, m^c := m_t                               */
   int32_t lowrank_path;    /* ADAPM_PATH_*: which kernels run Algorithm 2's contractions           */
   uint64_t seed;           /* seeds L_0 in adapm_state_init                                        */
+  uint32_t flags;          /* ADAPM_FLAG_*; 0 = defaults                                           */
+  float   max_grad_norm;   /* global gradient clipping (Section 5.1: threshold 1.0): every gradient is
+                              multiplied by min(1, c / ||g||_2), the norm over all blocks; 0 or +inf = off */
+  int32_t tune_panels;     /* tensor path: 128-row panels per refit item (1..3); 0 = automatic     */
+  int32_t tune_stage_k;    /* tensor path: K per shared-memory stage (64 or 128); 0 = automatic    */
 } adapm_hparams;
 
 /* Library version (major*100 + minor). */
@@ -142,14 +166,30 @@ int adapm_state_init(adapm_ctx* ctx, void* state, adapm_stream stream);
 /* Learning rate eta_t of the next steps (Algorithm 1 takes a schedule; the caller owns it). */
 int adapm_set_lr(adapm_ctx* ctx, float lr);
 
-/* One optimizer step over all blocks; t is the 1-based step count (used by adam_debias only). */
+/*
+ * One optimizer step over all blocks (Algorithm 1, loop body); t is the 1-based step count.
+ * The tensor-core path keeps bf16 copies of the factors L, R in the workspace from one step to the
+ * next.  It rebuilds them from the state buffer when t is not the successor of the previous call's
+ * t, when the state or workspace pointer changed, after adapm_state_init and after
+ * adapm_state_changed; a caller who writes L or R in the state buffer between two consecutive steps
+ * (importing a checkpoint into the same buffer) must call adapm_state_changed.
+ */
 int adapm_step(adapm_ctx* ctx, void* params, const void* grads, void* state, int64_t t, adapm_stream stream);
+int adapm_state_changed(adapm_ctx* ctx);
+
+/*
+ * bf16 copy of the parameters (the weights a mixed-precision forward pass reads): every kernel that
+ * writes W also writes bf16(W), rounded to nearest even, at the same element offset of this buffer.
+ * bf16_dev_ptr: device, as many bf16 elements as params has floats, 256-B aligned; NULL turns it off.
+ * (Not part of Algorithm 1; saves the separate cast pass a training loop would run after the step.)
+ */
+int adapm_set_shadow_params(adapm_ctx* ctx, void* bf16_dev_ptr);
 
 /* Algorithmic HBM bytes of one step (every operand read once, every result written once). */
 size_t adapm_step_bytes(const adapm_ctx* ctx);
 /* Algorithmic flops of the low-rank contractions of one step: (4 K_eff + 4) m n r per block. */
 double adapm_step_flops(const adapm_ctx* ctx);
-/* Kernels adapm_step launches per call. */
+/* Kernels adapm_step launched in its last call (before the first call: in a steady-state step). */
 int64_t adapm_launch_count(const adapm_ctx* ctx);
 
 /*
@@ -162,8 +202,20 @@ int adapm_set_profiling(adapm_ctx* ctx, int32_t on);
 int adapm_get_launch_times(adapm_ctx* ctx, float* ms, int32_t* kinds, int64_t capacity, int64_t* n_out);
 const char* adapm_launch_kind_name(int32_t kind);
 
-/* Synchronise `stream`, read the device status word into *status (0 = fine) and clear it. */
+/* Synchronise `stream`, read the device status word into *status (0 = fine) and clear it.
+ * Bits: 1, 2 a shared-memory stage, 4, 8 an accumulator, 16 a parameter tile, 32 a team of CTAs was waited
+ * for too long; 64 a gradient was not finite and ADAPM_FLAG_CHECK_FINITE skipped the step (params and state
+ * are untouched: step again with good gradients).  Non-zero: returns ADAPM_EDEVICE (see the conventions above). */
 int adapm_get_status(adapm_ctx* ctx, adapm_stream stream, int32_t* status);
+
+/*
+ * Diagnostic (the paper has no counterpart): launches one CTA of the refit engine whose only work item
+ * waits for a team counter that nothing advances, with the wait limit cut to about a millisecond.
+ * The kernel must give up, set bit 32 of the status word and return; afterwards adapm_get_status
+ * reports ADAPM_EDEVICE once and the context keeps working.  Exercises the give-up path without
+ * faulting or hanging anything.
+ */
+int adapm_selftest_expired_wait(adapm_ctx* ctx, adapm_stream stream);
 
 /*
  * Stand-alone block-mean of g^2 (the reduction behind ADAPM_V_BLOCKMEAN; Adam-mini combination):

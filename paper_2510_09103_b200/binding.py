@@ -17,6 +17,8 @@ V_ELEMENT, V_BLOCKMEAN = 0, 1
 GRAD_F32, GRAD_BF16 = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 STATE_M, STATE_L, STATE_R, STATE_V = 0, 1, 2, 3
+FLAG_NO_PANEL_TEAMS, FLAG_FORCE_PANEL_TEAMS, FLAG_NO_SUMSQ_FOLD, FLAG_CHECK_FINITE = 1, 2, 4, 8
+ST_WAIT_TEAM, ST_NONFINITE_GRAD = 32, 64
 
 EXPORTS = (
     "adapm_version", "adapm_strerror", "adapm_last_cuda_error", "adapm_plan_default", "adapm_create",
@@ -24,7 +26,7 @@ EXPORTS = (
     "adapm_workspace_bytes", "adapm_set_workspace", "adapm_state_init", "adapm_set_lr", "adapm_step",
     "adapm_step_bytes", "adapm_step_flops", "adapm_launch_count", "adapm_get_status",
     "adapm_group_meansq_scratch_bytes", "adapm_group_meansq", "adapm_set_profiling", "adapm_get_launch_times",
-    "adapm_launch_kind_name", "adapm_group_meansq_static",
+    "adapm_launch_kind_name", "adapm_group_meansq_static", "adapm_state_changed", "adapm_selftest_expired_wait", "adapm_set_shadow_params",
 )
 
 
@@ -49,13 +51,15 @@ class adapm_hparams(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("clip", C.c_float), ("inner_iters", C.c_int32), ("inner_lr_scale", C.c_float),
                 ("grad_dtype", C.c_int32), ("adam_debias", C.c_int32), ("correction", C.c_int32),
-                ("lowrank_path", C.c_int32), ("seed", C.c_uint64)]
+                ("lowrank_path", C.c_int32), ("seed", C.c_uint64), ("flags", C.c_uint32),
+                ("max_grad_norm", C.c_float), ("tune_panels", C.c_int32), ("tune_stage_k", C.c_int32)]
 
 
 def hparams(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, clip=1.0, inner_iters=5, inner_lr_scale=1.0,
-            grad_dtype=GRAD_BF16, adam_debias=0, correction=1, lowrank_path=PATH_AUTO, seed=0) -> adapm_hparams:
+            grad_dtype=GRAD_BF16, adam_debias=0, correction=1, lowrank_path=PATH_AUTO, seed=0, flags=0,
+            max_grad_norm=0.0, tune_panels=0, tune_stage_k=0) -> adapm_hparams:
     return adapm_hparams(lr, beta1, beta2, eps, clip, inner_iters, inner_lr_scale, grad_dtype, adam_debias,
-                         correction, lowrank_path, seed)
+                         correction, lowrank_path, seed, flags, max_grad_norm, tune_panels, tune_stage_k)
 
 
 class AdapmError(RuntimeError):
@@ -108,6 +112,9 @@ def load(build_if_missing: bool = True) -> C.CDLL:
         "adapm_set_profiling": (C.c_int, [vp, i32]),
         "adapm_get_launch_times": (C.c_int, [vp, C.POINTER(C.c_float), C.POINTER(i32), i64, C.POINTER(i64)]),
         "adapm_launch_kind_name": (C.c_char_p, [i32]),
+        "adapm_state_changed": (C.c_int, [vp]),
+        "adapm_selftest_expired_wait": (C.c_int, [vp, vp]),
+        "adapm_set_shadow_params": (C.c_int, [vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -225,6 +232,16 @@ class Context:
     def adapm_step(self, params, grads, state, t: int, stream=None) -> None:
         _check(self._lib.adapm_step(self._h, _ptr(params), _ptr(grads), _ptr(state), t, _stream(stream)),
                "adapm_step")
+
+    def adapm_set_shadow_params(self, buf) -> None:
+        _check(self._lib.adapm_set_shadow_params(self._h, _ptr(buf)), "adapm_set_shadow_params")
+        self._shadow = buf             # keep the caller's buffer alive
+
+    def adapm_state_changed(self) -> None:
+        _check(self._lib.adapm_state_changed(self._h), "adapm_state_changed")
+
+    def adapm_selftest_expired_wait(self, stream=None) -> None:
+        _check(self._lib.adapm_selftest_expired_wait(self._h, _stream(stream)), "adapm_selftest_expired_wait")
 
     def adapm_step_bytes(self) -> int:
         return self._lib.adapm_step_bytes(self._h)

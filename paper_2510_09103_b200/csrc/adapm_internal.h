@@ -33,7 +33,10 @@ inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 enum Base : int32_t { BASE_NONE = -1, BASE_PARAMS = 0, BASE_GRADS = 1, BASE_STATE = 2, BASE_WORK = 3 };
 
 struct Bases {
-  void* p[4];   // params (fp32), grads (fp32 | bf16), state (fp32), workspace (bytes; offsets in floats)
+  void* p[4];             // params (fp32), grads (fp32 | bf16), state (fp32), workspace (bytes; offsets in floats)
+  const int32_t* status;  // device status word: a kernel that finds it set writes nothing
+  const float* gscale;    // device scalars {s, s^2}: every gradient counts as s g (global norm clipping); null: 1
+  uint16_t* shadow;       // bf16 copy of the parameters, written wherever W is written; null: none
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -129,30 +132,45 @@ struct StepScalars {
 // one launch of the static per-step program
 enum LaunchKind : int32_t {
   LK_REDUCE_PARTIAL, LK_REDUCE_FINAL, LK_STREAM, LK_GEMM, LK_APPLY_SIMT, LK_COMMIT,
-  LK_TC_CONVERT, LK_TC_GRAM, LK_TC_PANEL, LK_TC_APPLY
+  LK_TC_CONVERT, LK_TC_GRAM, LK_TC_PANEL, LK_TC_APPLY,
+  LK_REDUCE_ROWS,       // reduce_final over the row sums of g^2 that the first refit pass left
+  LK_GRADNORM           // global gradient norm and the clip factor
+};
+// when a launch of the program runs
+enum LaunchWhen : int32_t {
+  WHEN_ALWAYS = 0,
+  WHEN_EVEN, WHEN_ODD   // only in steps of that parity (the factor sets swap roles from step to step)
 };
 struct Launch {
   LaunchKind kind;
   int64_t table_off;    // byte offset of its descriptor table in the device table blob
   int64_t n_items;      // descriptors
   int64_t grid;         // CTAs
-  int64_t aux0 = 0, aux1 = 0, aux2 = 0, aux3 = 0;
+  int64_t aux0 = 0, aux1 = 0, aux2 = 0, aux3 = 0, aux4 = 0, aux5 = 0;
+  int32_t when = WHEN_ALWAYS;
+  int32_t only_convert = 0;   // 1: only in a step that rebuilds the split copies of the factors
 };
 
 // ---------------------------------------------------------------------------------------------
 // kernel launchers (defined in the .cu files)
 // ---------------------------------------------------------------------------------------------
+// `status` is the device status word: a kernel that finds it set writes nothing (an earlier launch gave up).
 int launch_stream(const StreamBlk* d_tab, const int32_t* d_cta_blk, int64_t grid, const Bases& b,
                   const StepScalars& sc, int grad_dtype, cudaStream_t s);
 int launch_reduce_partial(const ReduceJob* d_tab, const int32_t* d_cta_job, int64_t n_jobs, int64_t n_units, const void* grads,
-                          float* work, int grad_dtype, cudaStream_t s);
+                          float* work, int grad_dtype, const int32_t* status, cudaStream_t s);
 int launch_reduce_final(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_groups, float* state, const float* work,
-                        float beta2, cudaStream_t s);
+                        float beta2, const int32_t* status, const float* gscale, cudaStream_t s);
+// global gradient norm: per-chunk sums of g^2 over every block, then {s, s^2} = clip factor into gscale
+struct NormRange { int64_t off, numel, first_cta; };
+constexpr int kNormChunk = 16384;
+int launch_gradnorm(const NormRange* d_tab, const int32_t* d_cta_range, int64_t n_ctas, const void* grads, int grad_dtype,
+                    float* partials, float max_norm, int check_finite, float* gscale, int32_t* status, cudaStream_t s);
 int launch_gemm(const GemmProb* d_tab, int64_t n_prob, int64_t n_tiles, const Bases& b, int grad_dtype,
                 cudaStream_t s);
 int launch_apply_simt(const ApplyBlk* d_tab, int64_t n_blk, int64_t n_tiles, const Bases& b, const StepScalars& sc,
                       int grad_dtype, cudaStream_t s);
-int launch_copy_f32(float* dst, const float* src, int64_t n, cudaStream_t s);
+int launch_copy_f32(float* dst, const float* src, int64_t n, const int32_t* status, cudaStream_t s);
 int launch_meansq_partial(const void* g, int grad_dtype, int64_t n_groups, int64_t group_elems, int chunks_per_group,
                           float* partial, cudaStream_t s);
 int launch_meansq_final(const float* partial, int64_t n_groups, int64_t group_elems, int chunks_per_group, float* out,
@@ -194,6 +212,13 @@ struct adapm_ctx {
   // optional per-launch timing (adapm_set_profiling)
   int profiling = 0, prof_valid = 0;
   std::vector<cudaEvent_t> prof_events;
+  std::vector<int32_t> prof_kinds;     // kinds of the launches the last profiled step issued, in order
+  int64_t last_step_launches = 0;      // kernels the last adapm_step launched
+
+  float* d_gscale = nullptr;           // device scalars {s, s^2}: the step's clip factor (global norm clipping), or null
+  void* shadow = nullptr;              // caller's bf16 copy of the parameters (adapm_set_shadow_params), or null
+  int use_gscale = 0;                  // the program starts with the gradient-norm pass
+  unsigned char* d_probe = nullptr;    // item table of the expired-wait probe
 
   size_t step_bytes = 0;
   double step_flops = 0;

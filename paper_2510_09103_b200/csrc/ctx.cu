@@ -36,6 +36,9 @@ int validate(const adapm_block* blocks, int64_t n, const adapm_hparams& hp) {
   if (!std::isfinite(hp.lr) || !std::isfinite(hp.inner_lr_scale)) return ADAPM_EINVAL;
   if (hp.grad_dtype != ADAPM_GRAD_F32 && hp.grad_dtype != ADAPM_GRAD_BF16) return ADAPM_EINVAL;
   if (hp.lowrank_path < ADAPM_PATH_AUTO || hp.lowrank_path > ADAPM_PATH_TENSOR) return ADAPM_EINVAL;
+  if (!(hp.max_grad_norm >= 0.f)) return ADAPM_ERANGE;      // 0 and +inf both mean "no clipping"; NaN is refused
+  if (hp.tune_panels < 0 || hp.tune_panels > 3) return ADAPM_ERANGE;
+  if (hp.tune_stage_k != 0 && hp.tune_stage_k != 64 && hp.tune_stage_k != 128) return ADAPM_ERANGE;
   std::vector<std::pair<int64_t, int64_t>> spans;
   spans.reserve((size_t)n);
   for (int64_t i = 0; i < n; ++i) {
@@ -67,10 +70,14 @@ int validate(const adapm_block* blocks, int64_t n, const adapm_hparams& hp) {
 // the tensor-core program of the low-rank blocks; defined in lowrank_tc.cu
 bool tensor_path_block_ok(const adapm_hparams& hp, const adapm_block& b);
 int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const std::vector<double>& etas,
-                         int64_t& work_cursor);
-int tensor_prepare_step(adapm_ctx* c, const Bases& b, cudaStream_t s);
-int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepScalars& sc, cudaStream_t s);
+                         int64_t& work_cursor, std::vector<ReduceJob>& row_jobs, int64_t& row_groups);
+int tensor_prepare_step(adapm_ctx* c, const Bases& b, int64_t t, cudaStream_t s, int* parity, int* convert);
+int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepScalars& sc, int parity,
+                      cudaStream_t s);
 void destroy_tensor_program(adapm_ctx* c);
+void tensor_state_changed(adapm_ctx* c);
+int run_expired_wait_probe(adapm_ctx* c, cudaStream_t s);
+size_t probe_table(std::vector<unsigned char>& out);
 
 }  // namespace adapm
 
@@ -199,8 +206,11 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     sblk.push_back(s);
   }
 
-  // group sums of g^2 of the low-rank blocks come from the reduction kernels
+  // Group sums of g^2 of the low-rank blocks come from the reduction kernels, except on the tensor path when
+  // there is a refit pass: its row panels read every row of g anyway and leave the row sums behind.
+  const bool fold_sumsq = K_eff > 0 && !(hp->flags & ADAPM_FLAG_NO_SUMSQ_FOLD);
   for (int pass = 0; pass < 2; ++pass) {
+    if (pass == 1 && fold_sumsq) break;
     for (int64_t i : (pass == 0 ? lowrank_ids : tc_ids)) {
       const adapm_block& b = c->blocks[i];
       if (b.v_mode != ADAPM_V_BLOCKMEAN) continue;
@@ -211,6 +221,25 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   }
 
   auto& prog = c->program;
+  // Global gradient-norm clipping (and the finite check, which rides on the same reduction) needs the norm of
+  // every gradient before anything uses one: a pass of its own over g.
+  const bool clip_on = hp->max_grad_norm > 0.f && std::isfinite(hp->max_grad_norm);
+  if (clip_on || (hp->flags & ADAPM_FLAG_CHECK_FINITE)) {
+    std::vector<NormRange> ranges;
+    std::vector<int32_t> cta_range;
+    for (int i = 0; i < n; ++i) {
+      const adapm_block& b = c->blocks[i];
+      NormRange r{b.offset, (int64_t)b.rows * b.cols, (int64_t)cta_range.size()};
+      for (int64_t q = 0; q < (r.numel + kNormChunk - 1) / kNormChunk; ++q) cta_range.push_back((int32_t)ranges.size());
+      ranges.push_back(r);
+    }
+    Launch GN{LK_GRADNORM, append_table(c->h_tables, ranges), (int64_t)ranges.size(), (int64_t)cta_range.size()};
+    GN.aux0 = append_table(c->h_tables, cta_range);
+    GN.aux1 = work_cursor;                                   // per-chunk sums
+    work_cursor += round_up((int64_t)cta_range.size(), kStateAlign);
+    prog.push_back(GN);
+    c->use_gscale = 1;
+  }
   if (!rjobs.empty()) {
     const int64_t off = append_table(c->h_tables, rjobs);
     // CTA index -> job of the CTA's first unit (the job table is sorted by first_unit), so that a warp finds its job
@@ -247,8 +276,17 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     c->n_init_jobs = (int64_t)ijobs.size();
   }
   if (!tc_ids.empty()) {
-    rc = build_tensor_program(c, tc_ids, etas, work_cursor);
+    std::vector<ReduceJob> row_jobs;
+    int64_t row_groups = 0;
+    rc = build_tensor_program(c, tc_ids, etas, work_cursor, row_jobs, row_groups);
     if (rc != ADAPM_OK) { adapm_destroy(c); return rc; }
+    if (!row_jobs.empty()) {
+      const int64_t off = append_table(c->h_tables, row_jobs);
+      for (Launch& L : prog)
+        if (L.kind == LK_REDUCE_ROWS) {
+          L.table_off = off; L.n_items = (int64_t)row_jobs.size(); L.grid = (row_groups + 7) / 8; L.aux0 = row_groups;
+        }
+    }
   }
   if (!lowrank_ids.empty()) {
     // workspace: two copies of the [L,R] section (ping-pong iterates), A/B with the same layout, Gram matrices
@@ -363,6 +401,17 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     e = cudaMemcpy(c->d_tables, c->h_tables.data(), c->h_tables.size(), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_status, 256);
   if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, 256);
+  if (e == cudaSuccess && c->use_gscale) {
+    const float ones[2] = {1.f, 1.f};
+    e = cudaMalloc((void**)&c->d_gscale, 256);
+    if (e == cudaSuccess) e = cudaMemcpy(c->d_gscale, ones, sizeof(ones), cudaMemcpyHostToDevice);
+  }
+  {
+    std::vector<unsigned char> probe;
+    const size_t pb = probe_table(probe);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_probe, pb);
+    if (e == cudaSuccess) e = cudaMemcpy(c->d_probe, probe.data(), pb, cudaMemcpyHostToDevice);
+  }
   if (e != cudaSuccess) {
     set_cuda_error(e, "adapm_create upload");
     adapm_destroy(c);
@@ -378,6 +427,8 @@ extern "C" void adapm_destroy(adapm_ctx* c) {
   for (auto e : c->prof_events) if (e) cudaEventDestroy(e);
   if (c->d_tables) cudaFree(c->d_tables);
   if (c->d_status) cudaFree(c->d_status);
+  if (c->d_probe) cudaFree(c->d_probe);
+  if (c->d_gscale) cudaFree(c->d_gscale);
   delete c;
 }
 
@@ -428,6 +479,7 @@ extern "C" int adapm_state_init(adapm_ctx* c, void* state, adapm_stream stream) 
   if ((uintptr_t)state % 256) return ADAPM_EALIGN;
   cudaStream_t s = (cudaStream_t)stream;
   ADAPM_CUDA(cudaMemsetAsync(state, 0, (size_t)c->state_floats * 4, s));
+  tensor_state_changed(c);
   if (c->n_init_jobs > 0)
     return launch_init_L0((const InitJob*)(c->d_tables + c->init_table_off), c->n_init_jobs, (float*)state, c->hp.seed, s);
   return ADAPM_OK;
@@ -441,7 +493,32 @@ extern "C" int adapm_set_lr(adapm_ctx* c, float lr) {
 
 extern "C" size_t adapm_step_bytes(const adapm_ctx* c) { return c ? c->step_bytes : 0; }
 extern "C" double adapm_step_flops(const adapm_ctx* c) { return c ? c->step_flops : 0.0; }
-extern "C" int64_t adapm_launch_count(const adapm_ctx* c) { return c ? (int64_t)c->program.size() : 0; }
+extern "C" int64_t adapm_launch_count(const adapm_ctx* c) {
+  if (!c) return 0;
+  if (c->last_step_launches > 0) return c->last_step_launches;
+  int64_t n = 0;
+  for (const Launch& L : c->program)
+    if ((L.when == WHEN_ALWAYS || L.when == WHEN_EVEN) && !L.only_convert) ++n;
+  return n;
+}
+
+extern "C" int adapm_set_shadow_params(adapm_ctx* c, void* bf16_dev_ptr) {
+  if (!c) return ADAPM_EINVAL;
+  if ((uintptr_t)bf16_dev_ptr % 256) return ADAPM_EALIGN;
+  c->shadow = bf16_dev_ptr;
+  return ADAPM_OK;
+}
+
+extern "C" int adapm_state_changed(adapm_ctx* c) {
+  if (!c) return ADAPM_EINVAL;
+  tensor_state_changed(c);
+  return ADAPM_OK;
+}
+
+extern "C" int adapm_selftest_expired_wait(adapm_ctx* c, adapm_stream stream) {
+  if (!c) return ADAPM_EINVAL;
+  return run_expired_wait_probe(c, (cudaStream_t)stream);
+}
 
 extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* state, int64_t t, adapm_stream stream) {
   if (!c || !params || !grads || !state || t < 1) return ADAPM_EINVAL;
@@ -468,25 +545,40 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
   Bases b;
   b.p[BASE_PARAMS] = params; b.p[BASE_GRADS] = const_cast<void*>(grads); b.p[BASE_STATE] = state;
   b.p[BASE_WORK] = c->workspace;
+  b.status = c->d_status; b.gscale = c->d_gscale; b.shadow = (uint16_t*)c->shadow;
   float* work = (float*)c->workspace;
 
+  int parity = 0, convert = 0;
   if (c->tc) {
-    const int prc = tensor_prepare_step(c, b, s);
+    const int prc = tensor_prepare_step(c, b, t, s, &parity, &convert);
     if (prc != ADAPM_OK) return prc;
   }
   const bool prof = c->profiling && c->prof_events.size() == c->program.size() + 1;
-  if (prof) ADAPM_CUDA(cudaEventRecord(c->prof_events[0], s));
+  if (prof) {
+    c->prof_kinds.clear();
+    ADAPM_CUDA(cudaEventRecord(c->prof_events[0], s));
+  }
   size_t li = 0;
   for (const Launch& L : c->program) {
+    if ((L.only_convert && !convert) || (L.when == WHEN_EVEN && parity != 0) || (L.when == WHEN_ODD && parity != 1))
+      continue;
     const unsigned char* tab = c->d_tables + L.table_off;
     int rc = ADAPM_OK;
     switch (L.kind) {
+      case LK_GRADNORM:
+        rc = launch_gradnorm((const NormRange*)tab, (const int32_t*)(c->d_tables + L.aux0), L.grid, grads, hp.grad_dtype,
+                             work + L.aux1, std::isfinite(hp.max_grad_norm) ? hp.max_grad_norm : 0.f,
+                             (hp.flags & ADAPM_FLAG_CHECK_FINITE) ? 1 : 0, c->d_gscale, c->d_status, s);
+        break;
       case LK_REDUCE_PARTIAL:
         rc = launch_reduce_partial((const ReduceJob*)tab, (const int32_t*)(c->d_tables + L.aux1), L.n_items, L.aux0, grads,
-                                   work, hp.grad_dtype, s);
+                                   work, hp.grad_dtype, c->d_status, s);
         break;
       case LK_REDUCE_FINAL:
-        rc = launch_reduce_final((const ReduceJob*)tab, L.n_items, L.aux0, (float*)state, work, hp.beta2, s); break;
+      case LK_REDUCE_ROWS:
+        rc = launch_reduce_final((const ReduceJob*)tab, L.n_items, L.aux0, (float*)state, work, hp.beta2, c->d_status,
+                                 c->d_gscale, s);
+        break;
       case LK_STREAM:
         rc = launch_stream((const StreamBlk*)tab, (const int32_t*)(c->d_tables + L.aux0), L.grid, b, sc, hp.grad_dtype, s);
         break;
@@ -495,14 +587,18 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
       case LK_APPLY_SIMT:
         rc = launch_apply_simt((const ApplyBlk*)tab, L.n_items, L.grid, b, sc, hp.grad_dtype, s); break;
       case LK_COMMIT:
-        rc = launch_copy_f32((float*)state, work + c->ws_lr[c->final_lr_buf], c->lr_section_floats, s); break;
+        rc = launch_copy_f32((float*)state, work + c->ws_lr[c->final_lr_buf], c->lr_section_floats, c->d_status, s); break;
       default:
-        rc = run_tensor_launch(c, L, b, sc, s); break;
+        rc = run_tensor_launch(c, L, b, sc, parity, s); break;
     }
     if (rc != ADAPM_OK) return rc;
     ++li;
-    if (prof) ADAPM_CUDA(cudaEventRecord(c->prof_events[li], s));
+    if (prof) {
+      c->prof_kinds.push_back((int32_t)L.kind);
+      ADAPM_CUDA(cudaEventRecord(c->prof_events[li], s));
+    }
   }
+  c->last_step_launches = (int64_t)li;
   if (prof) c->prof_valid = 1;
   return ADAPM_OK;
 }
@@ -520,14 +616,16 @@ extern "C" int adapm_set_profiling(adapm_ctx* c, int32_t on) {
 
 extern "C" int adapm_get_launch_times(adapm_ctx* c, float* ms, int32_t* kinds, int64_t capacity, int64_t* n_out) {
   if (!c || !n_out) return ADAPM_EINVAL;
-  *n_out = (int64_t)c->program.size();
+  // the launches of the last profiled step (a step runs a subset of the program: see LaunchWhen)
+  const size_t n = c->prof_valid ? c->prof_kinds.size() : c->program.size();
+  *n_out = (int64_t)n;
   if (!ms && !kinds) return ADAPM_OK;
-  if (capacity < (int64_t)c->program.size()) return ADAPM_ERANGE;
+  if (capacity < (int64_t)n) return ADAPM_ERANGE;
   if (!c->prof_valid) return ADAPM_EINVAL;
-  ADAPM_CUDA(cudaEventSynchronize(c->prof_events.back()));
-  for (size_t i = 0; i < c->program.size(); ++i) {
+  ADAPM_CUDA(cudaEventSynchronize(c->prof_events[n]));
+  for (size_t i = 0; i < n; ++i) {
     if (ms) ADAPM_CUDA(cudaEventElapsedTime(&ms[i], c->prof_events[i], c->prof_events[i + 1]));
-    if (kinds) kinds[i] = (int32_t)c->program[i].kind;
+    if (kinds) kinds[i] = c->prof_kinds[i];
   }
   return ADAPM_OK;
 }
@@ -536,6 +634,8 @@ extern "C" const char* adapm_launch_kind_name(int32_t kind) {
   switch (kind) {
     case LK_REDUCE_PARTIAL: return "reduce_partial";
     case LK_REDUCE_FINAL: return "reduce_final";
+    case LK_REDUCE_ROWS: return "reduce_rows";
+    case LK_GRADNORM: return "grad_norm";
     case LK_STREAM: return "stream_update";
     case LK_GEMM: return "gemm_simt";
     case LK_APPLY_SIMT: return "apply_simt";

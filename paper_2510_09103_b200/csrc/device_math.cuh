@@ -70,6 +70,13 @@ __device__ __forceinline__ void store8f(float* p, const float* f) {
   *(reinterpret_cast<float4*>(p) + 1) = make_float4(f[4], f[5], f[6], f[7]);
 }
 
+// two floats -> packed bf16 pair, round to nearest even (x0 in the low half)
+__device__ __forceinline__ uint32_t pack_bf16x2(float x0, float x1) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(x1), "f"(x0));
+  return d;
+}
+
 // Algorithm 1 line 9: W - lr s_b ( clamp(m^c / (sqrt(v) + eps)) + lambda_b W ).
 // Comparisons (not fminf/fmaxf) so that a NaN ratio stays NaN.
 __device__ __forceinline__ float adapm_param_update(float w, float mc, float v, const StepScalars& sc, float lr_s,

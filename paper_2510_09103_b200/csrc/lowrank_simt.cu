@@ -71,8 +71,13 @@ __global__ void __launch_bounds__(256) gemm_kernel(const GemmProb* __restrict__ 
   __shared__ __align__(16) float Xs[TK][TM + 4];
   __shared__ __align__(16) float Ys[TK][TN + 4];
   __shared__ GemmProb sP;
-  if (threadIdx.x == 0) sP = find_by_first_tile(tab, n_prob, (int64_t)blockIdx.x);
+  __shared__ int skip;
+  if (threadIdx.x == 0) {
+    sP = find_by_first_tile(tab, n_prob, (int64_t)blockIdx.x);
+    skip = *b.status != 0;
+  }
   __syncthreads();
+  if (skip) return;
   const GemmProb& P = sP;
   const int64_t tile = (int64_t)blockIdx.x - P.first_tile;
   const int i0 = (int)(tile / P.tiles_n) * TM, j0 = (int)(tile % P.tiles_n) * TN;
@@ -88,6 +93,8 @@ __global__ void __launch_bounds__(256) gemm_kernel(const GemmProb* __restrict__ 
   const float* Z1 = P.z1_base >= 0 ? static_cast<const float*>(b.p[P.z1_base]) + P.z1_off : nullptr;
   const float* Z2 = P.z2_base >= 0 ? static_cast<const float*>(b.p[P.z2_base]) + P.z2_off : nullptr;
   const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+  // a product with the gradient as an operand is a product with the clipped gradient
+  const float gprod = (b.gscale && (P.x_base == BASE_GRADS || P.y_base == BASE_GRADS)) ? __ldg(b.gscale) : 1.f;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int i = i0 + ty * 4 + r;
@@ -97,7 +104,7 @@ __global__ void __launch_bounds__(256) gemm_kernel(const GemmProb* __restrict__ 
       const int j = j0 + tx * 4 + c;
       if (j >= P.N) continue;
       const int64_t o = (int64_t)i * P.ldc + j;
-      float x = P.alpha * acc[r][c];
+      float x = (P.alpha * gprod) * acc[r][c];
       if (P.beta != 0.f) x += P.beta * C[o];
       if (Z1) x += P.c1 * Z1[o];
       if (Z2) x += P.c2 * Z2[o];
@@ -112,9 +119,16 @@ __global__ void __launch_bounds__(256) apply_simt_kernel(const ApplyBlk* __restr
   __shared__ __align__(16) float Xs[TK][TM + 4];
   __shared__ __align__(16) float Ys[TK][TN + 4];
   __shared__ ApplyBlk sA;
-  if (threadIdx.x == 0) sA = find_by_first_tile(tab, n_blk, (int64_t)blockIdx.x);
+  __shared__ int skip;
+  if (threadIdx.x == 0) {
+    sA = find_by_first_tile(tab, n_blk, (int64_t)blockIdx.x);
+    skip = *b.status != 0;
+  }
   __syncthreads();
+  if (skip) return;
   const ApplyBlk& A = sA;
+  const float gs = b.gscale ? __ldg(b.gscale) : 1.f;
+  uint16_t* shadow = b.shadow ? b.shadow + A.off : nullptr;
   const int64_t tile = (int64_t)blockIdx.x - A.first_tile;
   const int i0 = (int)(tile / A.tiles_n) * TM, j0 = (int)(tile % A.tiles_n) * TN;
   const int m = A.rows, n = A.cols, r = A.rank;
@@ -145,14 +159,16 @@ __global__ void __launch_bounds__(256) apply_simt_kernel(const ApplyBlk* __restr
       const int j = j0 + tx * 4 + c;
       if (j >= n) continue;
       const int64_t o = (int64_t)i * n + j;
-      const float g = load_operand<BF16G>(G, true, o);
+      const float g = gs * load_operand<BF16G>(G, true, o);
       const float mc = sc.cg * g + sc.c0 * p0[rr][c] - sc.c1 * p1[rr][c];
       float v = v_row;
       if (A.v_mode == ADAPM_V_ELEMENT) {
         v = sc.beta2 * V[o] + (1.f - sc.beta2) * (g * g);
         V[o] = v;
       }
-      W[o] = adapm_param_update(W[o], mc, v, sc, lr_s, A.wd);
+      const float w_new = adapm_param_update(W[o], mc, v, sc, lr_s, A.wd);
+      W[o] = w_new;
+      if (shadow) shadow[o] = (uint16_t)(pack_bf16x2(w_new, 0.f) & 0xffffu);
     }
   }
 }

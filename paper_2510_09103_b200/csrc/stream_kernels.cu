@@ -34,7 +34,7 @@ __device__ __forceinline__ float team_sum(float x, float* smem8) {
 template <typename GT, int TEAM, bool HAS_M, bool HAS_V>
 __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float* __restrict__ params,
                                          const typename GT::elem* __restrict__ grads, float* __restrict__ state,
-                                         const StepScalars& sc, float* smem8) {
+                                         const StepScalars& sc, float* smem8, float gs, uint16_t* __restrict__ shadow) {
   const int lane = (TEAM == 32) ? (threadIdx.x & 31) : threadIdx.x;
 
   int64_t ustart, group;
@@ -99,7 +99,7 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
       __syncthreads();
       v_old = smem8[8];
     }
-    v_group = sc.beta2 * v_old + (1.f - sc.beta2) * (tot / (float)ulen);
+    v_group = sc.beta2 * v_old + (1.f - sc.beta2) * ((gs * gs) * (tot / (float)ulen));
     if (lane == 0) state[B.v_off + group] = v_group;
   } else if (B.v_mode == SV_GROUP_READY) {
     v_group = state[B.v_off + group];
@@ -147,6 +147,7 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
         GT::unpack(graw[c0 + b], gf);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
+          gf[i] *= gs;                       // the clipped gradient (gs = 1 without global clipping)
           float mc = gf[i];
           if (HAS_M) {
             m[b][i] = sc.beta1 * m[b][i] + a1 * gf[i];
@@ -159,6 +160,16 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
             float ratio = mc * k_ratio;
             ratio = ratio > sc.clip ? sc.clip : (ratio < -sc.clip ? -sc.clip : ratio);
             w[b][i] = w[b][i] - lr_s * (ratio + B.wd * w[b][i]);
+          }
+        }
+        if (shadow) {                        // bf16 copy of the new parameters
+          uint16_t* sp = shadow + B.off + ustart + e0;
+          if (full) {
+            *reinterpret_cast<uint4*>(sp) = make_uint4(pack_bf16x2(w[b][0], w[b][1]), pack_bf16x2(w[b][2], w[b][3]),
+                                                       pack_bf16x2(w[b][4], w[b][5]), pack_bf16x2(w[b][6], w[b][7]));
+          } else {
+            const int nval = ulen - e0 < 8 ? ulen - e0 : 8;
+            for (int i = 0; i < nval; ++i) sp[i] = (uint16_t)(pack_bf16x2(w[b][i], 0.f) & 0xffffu);
           }
         }
         if (full) {
@@ -181,14 +192,15 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
 template <typename GT, int TEAM>
 __device__ __forceinline__ void run_unit_any(const StreamBlk& B, int64_t unit, float* __restrict__ params,
                                              const typename GT::elem* __restrict__ grads, float* __restrict__ state,
-                                             const StepScalars& sc, float* smem8) {
+                                             const StepScalars& sc, float* smem8, float gs,
+                                             uint16_t* __restrict__ shadow) {
   const bool has_m = B.m_off >= 0, has_v = B.v_mode == SV_ELEMENT;
   if (has_m) {
-    if (has_v) run_unit<GT, TEAM, true, true>(B, unit, params, grads, state, sc, smem8);
-    else run_unit<GT, TEAM, true, false>(B, unit, params, grads, state, sc, smem8);
+    if (has_v) run_unit<GT, TEAM, true, true>(B, unit, params, grads, state, sc, smem8, gs, shadow);
+    else run_unit<GT, TEAM, true, false>(B, unit, params, grads, state, sc, smem8, gs, shadow);
   } else {
-    if (has_v) run_unit<GT, TEAM, false, true>(B, unit, params, grads, state, sc, smem8);
-    else run_unit<GT, TEAM, false, false>(B, unit, params, grads, state, sc, smem8);
+    if (has_v) run_unit<GT, TEAM, false, true>(B, unit, params, grads, state, sc, smem8, gs, shadow);
+    else run_unit<GT, TEAM, false, false>(B, unit, params, grads, state, sc, smem8, gs, shadow);
   }
 }
 
@@ -197,17 +209,24 @@ __global__ void __launch_bounds__(256, 2) stream_update_kernel(const StreamBlk* 
                                                                const int32_t* __restrict__ cta_blk,
                                                                float* __restrict__ params,
                                                                const typename GT::elem* __restrict__ grads,
-                                                               float* __restrict__ state, StepScalars sc) {
+                                                               float* __restrict__ state, StepScalars sc,
+                                                               const int32_t* __restrict__ status,
+                                                               const float* __restrict__ gscale,
+                                                               uint16_t* __restrict__ shadow) {
   __shared__ StreamBlk sB;
   __shared__ float smem8[12];
-  if (threadIdx.x == 0) sB = tab[cta_blk[blockIdx.x]];   // which block this CTA works on
+  if (threadIdx.x == 0) {
+    sB = tab[cta_blk[blockIdx.x]];                       // which block this CTA works on
+    if (*status != 0) sB.team = 0;                       // an earlier launch gave up: write nothing
+  }
   __syncthreads();
   const int64_t cta_local = (int64_t)blockIdx.x - sB.first_cta;
+  const float gs = gscale ? __ldg(gscale) : 1.f;
   if (sB.team == 32) {
     const int64_t unit = cta_local * 8 + (threadIdx.x >> 5);
-    if (unit < sB.n_units) run_unit_any<GT, 32>(sB, unit, params, grads, state, sc, smem8);
-  } else {
-    run_unit_any<GT, 256>(sB, cta_local, params, grads, state, sc, smem8);
+    if (unit < sB.n_units) run_unit_any<GT, 32>(sB, unit, params, grads, state, sc, smem8, gs, shadow);
+  } else if (sB.team == 256) {
+    run_unit_any<GT, 256>(sB, cta_local, params, grads, state, sc, smem8, gs, shadow);
   }
 }
 
@@ -240,9 +259,10 @@ __global__ void __launch_bounds__(256) reduce_partial_kernel(const ReduceJob* __
                                                              const int32_t* __restrict__ cta_job, int n_jobs,
                                                              int64_t n_units,
                                                              const typename GT::elem* __restrict__ grads,
-                                                             float* __restrict__ work) {
+                                                             float* __restrict__ work,
+                                                             const int32_t* __restrict__ status) {
   const int64_t unit = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (unit >= n_units) return;
+  if (unit >= n_units || *status != 0) return;
   int lo = cta_job[blockIdx.x];                       // job of the CTA's first unit; this warp's is at most 7 units on
   while (lo + 1 < n_jobs && tab[lo + 1].first_unit <= unit) ++lo;
   const ReduceJob J = tab[lo];
@@ -268,9 +288,11 @@ __device__ __forceinline__ float warp_sum_partials(const float* __restrict__ p, 
 
 __global__ void __launch_bounds__(256) reduce_final_kernel(const ReduceJob* __restrict__ tab, int n_jobs,
                                                            int64_t n_groups, float* __restrict__ state,
-                                                           const float* __restrict__ work, float beta2) {
+                                                           const float* __restrict__ work, float beta2,
+                                                           const int32_t* __restrict__ status,
+                                                           const float* __restrict__ gscale) {
   const int64_t gidx = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (gidx >= n_groups) return;
+  if (gidx >= n_groups || *status != 0) return;
   int lo = 0, hi = n_jobs - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
@@ -281,7 +303,8 @@ __global__ void __launch_bounds__(256) reduce_final_kernel(const ReduceJob* __re
   const float tot = warp_sum_partials(work + J.part_off + group * J.chunks_per_group, J.chunks_per_group);
   if ((threadIdx.x & 31) == 0) {
     float* v = state + J.v_off + group;
-    *v = beta2 * (*v) + (1.f - beta2) * (tot / (float)J.group_elems);
+    const float gs2 = gscale ? gscale[1] : 1.f;      // the sums are of the unclipped gradient
+    *v = beta2 * (*v) + (1.f - beta2) * (gs2 * (tot / (float)J.group_elems));
   }
 }
 
@@ -311,7 +334,76 @@ __global__ void __launch_bounds__(256) meansq_final_kernel(const float* __restri
   if ((threadIdx.x & 31) == 0) out[group] = tot / (float)group_elems;
 }
 
-__global__ void copy_f32_kernel(float4* __restrict__ dst, const float4* __restrict__ src, int64_t n4) {
+// ---- global gradient norm ---------------------------------------------------------------------------
+// Stage 1: one CTA per chunk of up to 16384 elements of one block; every thread adds its elements in a fixed
+// order, the warps and the CTA reduce in a fixed order.  Stage 2: one CTA adds the per-chunk sums in double,
+// again in a fixed order, and writes s = min(1, c / norm) and s^2.
+template <typename GT>
+__global__ void __launch_bounds__(256) gradnorm_partial_kernel(const NormRange* __restrict__ tab,
+                                                               const int32_t* __restrict__ cta_range,
+                                                               const typename GT::elem* __restrict__ grads,
+                                                               float* __restrict__ partials,
+                                                               const int32_t* __restrict__ status) {
+  __shared__ float warp_sums[8];
+  if (*status != 0) return;
+  const NormRange R = tab[cta_range[blockIdx.x]];
+  const int64_t start = ((int64_t)blockIdx.x - R.first_cta) * kNormChunk;
+  const int64_t rem = R.numel - start;
+  const int len = rem < kNormChunk ? (int)rem : kNormChunk;
+  const typename GT::elem* g = grads + R.off + start;
+  const int nchunks = (len + kChunkElems - 1) / kChunkElems;
+  float ss = 0.f;
+  for (int idx = threadIdx.x; idx < nchunks; idx += 256) {
+    const int e0 = idx * kChunkElems;
+    typename GT::raw8 r = (e0 + kChunkElems <= len) ? GT::load8(g + e0) : GT::load8_guarded(g + e0, len - e0);
+    float f[8];
+    GT::unpack(r, f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t += warp_sums[i];
+    partials[blockIdx.x] = t;
+  }
+}
+
+__global__ void __launch_bounds__(1024) gradnorm_final_kernel(const float* __restrict__ partials, int64_t n, float max_norm,
+                                                              int check_finite, float* __restrict__ gscale,
+                                                              int32_t* __restrict__ status) {
+  __shared__ double sums[1024];
+  if (*status != 0) return;
+  double t = 0.0;
+  for (int64_t i = threadIdx.x; i < n; i += 1024) t += (double)partials[i];
+  sums[threadIdx.x] = t;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) sums[threadIdx.x] += sums[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double total = sums[0];
+    float s = 1.f;
+    if (!(total >= 0.0) || total > 3.0e38) {           // NaN or Inf somewhere in the gradient
+      if (check_finite) atomicOr(status, 64);          // the rest of the step is skipped and the caller is told
+      else s = (float)(total - total);                 // NaN: propagates like any other NaN gradient
+    } else if (max_norm > 0.f && total > 0.0) {
+      const double norm = sqrt(total);
+      if (norm > (double)max_norm) s = (float)((double)max_norm / norm);
+    }
+    gscale[0] = s;
+    gscale[1] = s * s;
+  }
+}
+
+__global__ void copy_f32_kernel(float4* __restrict__ dst, const float4* __restrict__ src, int64_t n4,
+                                const int32_t* __restrict__ status) {
+  if (*status != 0) return;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x)
     dst[i] = src[i];
 }
@@ -333,32 +425,36 @@ int launch_stream(const StreamBlk* d_tab, const int32_t* d_cta_blk, int64_t grid
   if (grad_dtype == ADAPM_GRAD_BF16)
     stream_update_kernel<GradBF16><<<(unsigned)grid, 256, 0, s>>>(d_tab, d_cta_blk, (float*)b.p[BASE_PARAMS],
                                                                  (const uint16_t*)b.p[BASE_GRADS],
-                                                                 (float*)b.p[BASE_STATE], sc);
+                                                                 (float*)b.p[BASE_STATE], sc, b.status, b.gscale,
+                                                                 b.shadow);
   else
     stream_update_kernel<GradF32><<<(unsigned)grid, 256, 0, s>>>(d_tab, d_cta_blk, (float*)b.p[BASE_PARAMS],
                                                                 (const float*)b.p[BASE_GRADS],
-                                                                (float*)b.p[BASE_STATE], sc);
+                                                                (float*)b.p[BASE_STATE], sc, b.status, b.gscale,
+                                                                b.shadow);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }
 
 int launch_reduce_partial(const ReduceJob* d_tab, const int32_t* d_cta_job, int64_t n_jobs, int64_t n_units,
-                          const void* grads, float* work, int grad_dtype, cudaStream_t s) {
+                          const void* grads, float* work, int grad_dtype, const int32_t* status, cudaStream_t s) {
   if (n_units <= 0) return ADAPM_OK;
   const unsigned grid = (unsigned)((n_units + 7) / 8);
   if (grad_dtype == ADAPM_GRAD_BF16)
     reduce_partial_kernel<GradBF16><<<grid, 256, 0, s>>>(d_tab, d_cta_job, (int)n_jobs, n_units, (const uint16_t*)grads,
-                                                         work);
+                                                         work, status);
   else
-    reduce_partial_kernel<GradF32><<<grid, 256, 0, s>>>(d_tab, d_cta_job, (int)n_jobs, n_units, (const float*)grads, work);
+    reduce_partial_kernel<GradF32><<<grid, 256, 0, s>>>(d_tab, d_cta_job, (int)n_jobs, n_units, (const float*)grads, work,
+                                                        status);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }
 
 int launch_reduce_final(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_groups, float* state, const float* work,
-                        float beta2, cudaStream_t s) {
+                        float beta2, const int32_t* status, const float* gscale, cudaStream_t s) {
   if (n_groups <= 0) return ADAPM_OK;
-  reduce_final_kernel<<<(unsigned)((n_groups + 7) / 8), 256, 0, s>>>(d_tab, (int)n_jobs, n_groups, state, work, beta2);
+  reduce_final_kernel<<<(unsigned)((n_groups + 7) / 8), 256, 0, s>>>(d_tab, (int)n_jobs, n_groups, state, work, beta2,
+                                                                    status, gscale);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }
@@ -387,13 +483,28 @@ int launch_meansq_final(const float* partial, int64_t n_groups, int64_t group_el
   return ADAPM_OK;
 }
 
-int launch_copy_f32(float* dst, const float* src, int64_t n, cudaStream_t s) {
+int launch_gradnorm(const NormRange* d_tab, const int32_t* d_cta_range, int64_t n_ctas, const void* grads, int grad_dtype,
+                    float* partials, float max_norm, int check_finite, float* gscale, int32_t* status, cudaStream_t s) {
+  if (n_ctas <= 0) return ADAPM_OK;
+  if (grad_dtype == ADAPM_GRAD_BF16)
+    gradnorm_partial_kernel<GradBF16><<<(unsigned)n_ctas, 256, 0, s>>>(d_tab, d_cta_range, (const uint16_t*)grads, partials,
+                                                                      status);
+  else
+    gradnorm_partial_kernel<GradF32><<<(unsigned)n_ctas, 256, 0, s>>>(d_tab, d_cta_range, (const float*)grads, partials,
+                                                                     status);
+  ADAPM_LAUNCH_CHECK();
+  gradnorm_final_kernel<<<1, 1024, 0, s>>>(partials, n_ctas, max_norm, check_finite, gscale, status);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_copy_f32(float* dst, const float* src, int64_t n, const int32_t* status, cudaStream_t s) {
   if (n <= 0) return ADAPM_OK;
   // n is a multiple of 64 floats by construction of the state layout
   const int64_t n4 = n / 4;
   int64_t grid = (n4 + 255) / 256;
   if (grid > 148 * 16) grid = 148 * 16;
-  copy_f32_kernel<<<(unsigned)grid, 256, 0, s>>>((float4*)dst, (const float4*)src, n4);
+  copy_f32_kernel<<<(unsigned)grid, 256, 0, s>>>((float4*)dst, (const float4*)src, n4, status);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }

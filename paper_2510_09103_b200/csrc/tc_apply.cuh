@@ -19,6 +19,12 @@
 // accumulator row from tensor memory, its 16 columns of g and W from the (swizzled) buffer, and
 // puts the new W back in place.  A per-element v, where a block has one, travels like W.
 // The m x n matrices m_t, r_t and m^c are never stored.
+//
+// Ranks above 128 do not leave room for a resident L panel (4 rp columns of 128 rows).  The kernel's
+// second form (kStream) streams L as well: a stage of its ring holds four boxes - 64 columns of
+// L hi, L lo, R^T hi and R^T lo of one factor set - and feeds hi*hi, lo*hi and hi*lo for those
+// columns; the previous set is always taken first, the refitted set second.  Everything after the
+// accumulator (the g / W ring, the epilogue) is the same code.
 #pragma once
 
 #include <cuda.h>
@@ -43,6 +49,7 @@ struct ApplyItem {
   int64_t off;               // element offset of the block in params / grads
   int64_t v_off;             // float offset of v in state
   int32_t rows, cols, r, rp;
+  int32_t half;              // column at which the lo part of a factor set starts (a set is 2 half columns wide)
   int32_t map_l, map_r;      // split factors, previous and final set side by side: [rows, 4rp] and [cols, 4rp]
                              // = [hi0 | lo0 | hi1 | lo1], boxes of 64 x 128
   int32_t map_w, map_g;      // params and grads of the block, boxes of 32 x 128
@@ -62,6 +69,9 @@ struct ApplyArgs {
   int32_t* status;
   StepScalars sc;
   int32_t use_new;           // 0: c1 == 0, the refitted factors are not needed
+  int32_t parity;            // 0: the left half of the operands holds the previous factors, 1: the right half
+  const float* gscale;       // device scalar: every gradient counts as gscale[0] * g (nullptr: 1)
+  uint16_t* shadow;          // bf16 copy of the parameters, written with W (nullptr: none)
   int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
   int32_t n_rstages;         // R ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
   int32_t w_region_off;      // byte offset of the g / W ring
@@ -77,9 +87,14 @@ struct __align__(8) ApplyShared {
   int abort;
 };
 
+template <bool kStream>
 __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a) {
   extern __shared__ uint8_t dyn_smem[];
   __shared__ ApplyShared sh;
+  __shared__ int skip_launch;
+  if (threadIdx.x == 0) skip_launch = *reinterpret_cast<volatile int32_t*>(a.status) != 0;
+  __syncthreads();
+  if (skip_launch) return;   // an earlier launch of the step gave up: leave W and v untouched
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(dyn_smem) + 1023) & ~(uintptr_t)1023);
   uint8_t* smem_l = smem;
   uint8_t* smem_r = smem + a.r_region_off;
@@ -114,18 +129,42 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
       int l_loads = 0, r_loads = 0;
       for (int it = blockIdx.x; it < a.n_items && ok; it += gridDim.x) {
         const ApplyItem I = a.items[it];
+        if (kStream) {
+          // a stage = 64 columns of [L hi, L lo, R^T hi, R^T lo] of one set; previous set first
+          const int nbh = (I.rp + 63) >> 6;
+          for (int t = 0; t < I.n_tiles && ok; ++t) {
+            const int col0 = (I.tile0 + t) * kApplyNT;
+            for (int si = 0; si < n_sets && ok; ++si) {
+              const int xs = (si == 0 ? a.parity : 1 - a.parity) * 2 * I.half;
+              for (int jb = 0; jb < nbh; ++jb) {
+                if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
+                uint8_t* st = smem_r + (size_t)rs * (4 * kBoxBytes);
+                mbar_arrive_expect_tx(&sh.rfull[rs], 4u * kBoxBytes);
+                tma_load_box(st, a.maps + I.map_l, xs + 64 * jb, I.row0, &sh.rfull[rs]);
+                tma_load_box(st + kBoxBytes, a.maps + I.map_l, xs + I.half + 64 * jb, I.row0, &sh.rfull[rs]);
+                tma_load_box(st + 2 * kBoxBytes, a.maps + I.map_r, xs + 64 * jb, col0, &sh.rfull[rs]);
+                tma_load_box(st + 3 * kBoxBytes, a.maps + I.map_r, xs + I.half + 64 * jb, col0, &sh.rfull[rs]);
+                ++r_loads;
+                if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
+              }
+            }
+          }
+          continue;
+        }
         if (!mbar_wait(&sh.lempty, item_phase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
         const int nb = n_sets == 2 ? I.nbc2 : I.nbc1;
+        // with only the previous set in use, and that set in the right half, the boxes start there
+        const int x0 = (n_sets == 1 && a.parity) ? 2 * I.rp : 0;
         mbar_arrive_expect_tx(&sh.lfull, (uint32_t)nb * kBoxBytes);
         for (int bc = 0; bc < nb; ++bc)
-          tma_load_box(smem_l + (size_t)bc * kBoxBytes, a.maps + I.map_l, 64 * bc, I.row0, &sh.lfull);
+          tma_load_box(smem_l + (size_t)bc * kBoxBytes, a.maps + I.map_l, x0 + 64 * bc, I.row0, &sh.lfull);
         ++l_loads;
         for (int t = 0; t < I.n_tiles && ok; ++t) {
           const int col0 = (I.tile0 + t) * kApplyNT;
           for (int bc = 0; bc < nb; ++bc) {
             if (!mbar_wait(&sh.rempty[rs], rphase ^ 1u, abort, a.status, ST_WAIT_EMPTY)) { ok = false; break; }
             mbar_arrive_expect_tx(&sh.rfull[rs], (uint32_t)kBoxBytes);
-            tma_load_box(smem_r + (size_t)rs * kBoxBytes, a.maps + I.map_r, 64 * bc, col0, &sh.rfull[rs]);
+            tma_load_box(smem_r + (size_t)rs * kBoxBytes, a.maps + I.map_r, x0 + 64 * bc, col0, &sh.rfull[rs]);
             ++r_loads;
             if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
           }
@@ -162,6 +201,38 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
         const uint32_t idesc_pos = make_idesc(kApplyNT, false, false, false);
         const uint32_t idesc_neg = make_idesc(kApplyNT, false, false, true);
         const uint32_t la = desc_lo(l_base, 16);
+        if (kStream) {
+          const int nbh = (I.rp + 63) >> 6;
+          for (int t = 0; t < I.n_tiles && ok; ++t, ++j) {
+            const int acc = j & 1;
+            const uint32_t acc_phase = (uint32_t)(j >> 1) & 1u;
+            if (!mbar_wait(&sh.tempty[acc], acc_phase ^ 1u, abort, a.status, ST_WAIT_TMEM_EMPTY)) { ok = false; break; }
+            const uint32_t d = tmem_base + (uint32_t)(acc * kApplyNT);
+            uint32_t accumulate = 0;
+            for (int si = 0; si < n_sets && ok; ++si) {
+              const uint32_t idesc = si ? idesc_neg : idesc_pos;      // the refitted set enters negated
+              for (int jb = 0; jb < nbh; ++jb) {
+                if (!mbar_wait(&sh.rfull[rs], rphase, abort, a.status, ST_WAIT_FULL)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t st = r_base + (uint32_t)rs * (4u * kBoxBytes);
+                const uint32_t ahi = desc_lo(st, 16), alo = desc_lo(st + kBoxBytes, 16);
+                const uint32_t bhi = desc_lo(st + 2 * kBoxBytes, 16), blo = desc_lo(st + 3 * kBoxBytes, 16);
+                for (int kk = 0; kk < 4; ++kk) {
+                  if (4 * jb + kk >= ks) break;
+                  const uint32_t o = (uint32_t)(kk * 2);
+                  mma_bf16(d, desc_join(ahi + o, dhi), desc_join(bhi + o, dhi), idesc, accumulate);
+                  mma_bf16(d, desc_join(alo + o, dhi), desc_join(bhi + o, dhi), idesc, 1u);
+                  mma_bf16(d, desc_join(ahi + o, dhi), desc_join(blo + o, dhi), idesc, 1u);
+                  accumulate = 1;
+                }
+                mma_commit(&sh.rempty[rs]);
+                if (++rs == a.n_rstages) { rs = 0; rphase ^= 1u; }
+              }
+            }
+            if (ok) mma_commit(&sh.tfull[acc]);
+          }
+          continue;
+        }
         if (!mbar_wait(&sh.lfull, item_phase, abort, a.status, ST_WAIT_FULL)) break;
         for (int t = 0; t < I.n_tiles && ok; ++t, ++j) {
           const int acc = j & 1;
@@ -180,7 +251,8 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
               if (kb >= ktot) break;
               const int set = kb >= 2 * ks ? 1 : 0;
               const int w = kb - set * 2 * ks;         // K step inside the set: hi part, then lo part
-              const uint32_t idesc = set ? idesc_neg : idesc_pos;
+              // the set that holds the refitted factors enters with a negated A operand
+              const uint32_t idesc = (n_sets == 2 && (set ^ a.parity)) ? idesc_neg : idesc_pos;
               const uint64_t b = desc_join(rb + (uint32_t)(kk * 2), dhi);
               if (w < ks) {                            // hi * hi, lo * hi
                 mma_bf16(d, desc_join(la + kstep(kb), dhi), b, idesc, accumulate);
@@ -263,7 +335,9 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
     const int half = e >> 2;                              // which 16 columns of a quarter
     const uint32_t lane_addr = (uint32_t)(32 * wq4) << 16;
     const int rloc = 32 * wq4 + lane;                     // this thread's row of the panel
-    const StepScalars sc = a.sc;
+    StepScalars sc = a.sc;
+    const float gs = a.gscale ? *a.gscale : 1.f;
+    sc.cg *= gs;               // m^c = cg (gs g) + c0 D
     // byte offsets of this thread's 16-byte chunks inside a buffer: the 128-byte swizzle turns chunk c of
     // row r into chunk c ^ (r % 8), the 64-byte swizzle chunk c of a 64-byte row into c ^ ((r / 2) % 4)
     uint32_t w_at[4], g_at[2];
@@ -314,6 +388,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
             gf[8 * i + 2 * x + 1] = __uint_as_float(gw[x] & 0xffff0000u);
           }
         }
+        uint32_t shw[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float4* wp = reinterpret_cast<float4*>(buf + w_at[i]);
@@ -333,12 +408,23 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
               const float g1 = gf[4 * i + x];
-              vv[x] = sc.beta2 * vv[x] + (1.f - sc.beta2) * (g1 * g1);
+              vv[x] = sc.beta2 * vv[x] + (1.f - sc.beta2) * ((gs * g1) * (gs * g1));
               w[x] = adapm_param_update(w[x], sc.cg * g1 + sc.c0 * d[4 * i + x], vv[x], sc, lr_s, I.wd);
             }
             *vp = make_float4(vv[0], vv[1], vv[2], vv[3]);
           }
           *wp = make_float4(w[0], w[1], w[2], w[3]);
+          shw[2 * i] = pack_bf16x2(w[0], w[1]);
+          shw[2 * i + 1] = pack_bf16x2(w[2], w[3]);
+        }
+        if (a.shadow) {
+          // this thread's 16 columns of the row as bf16: two 16-byte stores (columns come in groups of 8)
+          const int col = (I.tile0 + (q >> 2)) * kApplyNT + sub * kApplyQC + 16 * half;
+          if (rok) {
+            uint16_t* sp = a.shadow + I.off + (int64_t)row * I.cols + col;
+            if (col < I.cols) *reinterpret_cast<uint4*>(sp) = make_uint4(shw[0], shw[1], shw[2], shw[3]);
+            if (col + 8 < I.cols) *reinterpret_cast<uint4*>(sp + 8) = make_uint4(shw[4], shw[5], shw[6], shw[7]);
+          }
         }
         // one arrival per warp: every lane orders its own writes (and tensor-memory reads), the warp meets
         fence_async_smem();

@@ -52,12 +52,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Waits for the phase with the given parity to complete.  Gives up after kSpinLimit polls or as
+// Waits for the phase with the given parity to complete.  Gives up after `limit` polls or as
 // soon as another thread of the CTA has given up (*abort != 0); then sets *abort, records `code` in
 // the device status word and returns false.  Callers leave their loops on false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
-                                          int32_t code) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+                                          int32_t code, uint32_t limit = kSpinLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 32) {
       __nanosleep(it > 4096 ? 256 : 32);

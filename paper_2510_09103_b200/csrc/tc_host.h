@@ -25,15 +25,15 @@ inline EncodeTiledFn encode_tiled_fn() {
 }
 
 // Tensor map of a row-major bf16 matrix [rows, cols] with row pitch `pitch_elems`, read in boxes of
-// 64 columns x 128 rows with the 128-byte swizzle; out-of-range elements read as zero.
+// 64 columns x box_rows rows with the 128-byte swizzle; out-of-range elements read as zero.
 // Requires: base 16-byte aligned, pitch a multiple of 8 elements.  Returns false on failure.
 inline bool encode_bf16_matrix(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
-                               uint64_t pitch_elems) {
+                               uint64_t pitch_elems, uint32_t box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {pitch_elems * 2};
-  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t box[2] = {64, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

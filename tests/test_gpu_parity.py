@@ -56,6 +56,14 @@ def test_llama60m_elementwise_v():
     _run(w, False, 6, sel=sample_blocks(blocks, 1))
 
 
+def test_gpt2_1p5b_4layers_elementwise_v():
+    """Rank 80 with a per-element v: the apply kernel's three-buffer form (v travels with W), followed by the oracle."""
+    w = WL.get_workload("gpt2_1p5b@4")
+    blocks, _ = A.adapm_plan_default(w.tensors, v_mode=A.V_ELEMENT)
+    sel = [i for i in sample_blocks(blocks, 1) if blocks[i].rows < 50000]
+    _run(w, False, 6, sel=sel, pooled=True, every=3)
+
+
 def test_gpt2_124m_sampled_blocks_20_steps():
     w = WL.get_workload("gpt2_124m")
     blocks, _ = A.adapm_plan_default(w.tensors)
@@ -295,15 +303,15 @@ def test_tensor_path_is_bitwise_reproducible():
     assert torch.equal(p1, p2) and torch.equal(s1, s2)
 
 
-def test_panel_team_schedule_changes_no_bit(monkeypatch):
+def test_panel_team_schedule_changes_no_bit():
     """The refit's panel launch hands its items to teams of CTAs kept in step by a counter when the set has enough
-    blocks (llama350m has); ADAPM_PANEL_TEAMS=0 hands them out longest-first instead.  Which CTA runs an item, and
-    when, must not change any result."""
+    blocks (llama350m has); ADAPM_FLAG_NO_PANEL_TEAMS hands them out longest-first instead.  Which CTA runs an
+    item, and when, must not change any result."""
     import torch
 
     def trajectory(teams):
-        monkeypatch.setenv("ADAPM_PANEL_TEAMS", teams)
-        run = ParityRun(WL.get_workload("llama350m"), True, oracle_blocks=[], lowrank_path=A.PATH_TENSOR)
+        run = ParityRun(WL.get_workload("llama350m"), True, oracle_blocks=[], lowrank_path=A.PATH_TENSOR,
+                        hp_overrides=dict(flags=0 if teams else A.FLAG_NO_PANEL_TEAMS))
         for _ in range(3):
             run.step()
         torch.cuda.synchronize()
@@ -312,9 +320,110 @@ def test_panel_team_schedule_changes_no_bit(monkeypatch):
         run.close()
         return out
 
-    p1, s1 = trajectory("1")
-    p0, s0 = trajectory("0")
+    p1, s1 = trajectory(True)
+    p0, s0 = trajectory(False)
     assert torch.equal(p1, p0) and torch.equal(s1, s0)
+
+
+@pytest.mark.parametrize("panels,stage_k", [(1, 128), (2, 64), (3, 64), (3, 128)])
+def test_tensor_path_engine_shapes(panels, stage_k):
+    """Every shape of the refit engine's pipeline - one to three panels per item, K = 64 or 128 per stage - against
+    the oracle, on blocks with ragged last panels and ranks that take each form of the epilogue."""
+    blocks = _pack([(700, 392, A.MOM_LOWRANK, 24, A.V_BLOCKMEAN, 1),
+                    (392, 1000, A.MOM_LOWRANK, 13, A.V_BLOCKMEAN, 8),
+                    (520, 136, A.MOM_LOWRANK, 40, A.V_ELEMENT, 0)])
+    w = WL.Workload("shapes", [], "bf16", "normal", steps=5)
+    _run(w, True, 5, path=A.PATH_TENSOR, blocks=blocks, hp=dict(tune_panels=panels, tune_stage_k=stage_k))
+
+
+def test_folded_row_sums_equal_the_separate_reduction_bit_for_bit_in_everything_but_v():
+    """The first refit pass adds up g^2 per row while it streams the gradient; ADAPM_FLAG_NO_SUMSQ_FOLD takes the
+    sums from a pass of its own instead.  The two add in different orders, so v may differ in the last bits (both
+    are checked against the oracle elsewhere); nothing else may change by more than that allows."""
+    import torch
+    blocks = _pack([(300, 256, A.MOM_LOWRANK, 20, A.V_BLOCKMEAN, 1), (128, 640, A.MOM_LOWRANK, 6, A.V_BLOCKMEAN, 0),
+                    (256, 512, A.MOM_LOWRANK, 16, A.V_BLOCKMEAN, 64)])
+
+    def trajectory(flags):
+        w = WL.Workload("fold", [], "bf16", "normal", steps=4)
+        run = ParityRun(w, True, lowrank_path=A.PATH_TENSOR, custom_blocks=blocks, hp_overrides=dict(flags=flags))
+        for _ in range(4):
+            run.step()
+            run.compare()
+        torch.cuda.synchronize()
+        out = run.params.clone(), run.state.clone()
+        assert run.ctx.adapm_get_status() == 0
+        run.close()
+        return out
+
+    p1, s1 = trajectory(0)
+    p0, s0 = trajectory(A.FLAG_NO_SUMSQ_FOLD)
+    assert torch.allclose(p1, p0, rtol=1e-5, atol=1e-9) and torch.allclose(s1, s0, rtol=1e-5, atol=1e-12)
+
+
+def test_tensor_path_resumes_bit_for_bit_and_follows_a_rewritten_state():
+    """The factor copies in the workspace carry over from step to step (the sets swap roles; nothing is converted).
+    A run that is exported after 3 steps and continued in a fresh context and workspace must equal an
+    uninterrupted one bit for bit, and a state buffer rewritten in place must be picked up after
+    adapm_state_changed."""
+    import torch
+    blocks = _pack([(300, 256, A.MOM_LOWRANK, 20, A.V_BLOCKMEAN, 1), (128, 640, A.MOM_LOWRANK, 6, A.V_ELEMENT, 0)])
+
+    def make():
+        return ParityRun(WL.Workload("resume", [], "bf16", "normal", steps=6), True, oracle_blocks=[],
+                         lowrank_path=A.PATH_TENSOR, custom_blocks=blocks)
+
+    def trajectory(split, in_place=False):
+        run = make()
+        for s in range(1, 7):
+            run.step()
+            if s == split and not in_place:
+                p, st, t = run.params.clone(), run.state.clone(), run.t
+                run.close()
+                run = make()
+                run.params.copy_(p); run.state.copy_(st); run.t = t
+            elif s == split:
+                # overwrite the state with itself through a copy and tell the library: the result must not move
+                st = run.state.clone()
+                run.state.zero_()
+                run.state.copy_(st)
+                run.ctx.adapm_state_changed()
+        torch.cuda.synchronize()
+        out = run.params.clone(), run.state.clone()
+        assert run.ctx.adapm_get_status() == 0
+        run.close()
+        return out
+
+    p1, s1 = trajectory(0)
+    p2, s2 = trajectory(3)
+    p3, s3 = trajectory(3, in_place=True)
+    assert torch.equal(p1, p2) and torch.equal(s1, s2)
+    assert torch.equal(p1, p3) and torch.equal(s1, s3)
+
+
+def test_an_expired_wait_is_reported_and_the_context_keeps_working():
+    """A wait inside the refit engine that can never be satisfied (a team counter nothing advances, with the limit
+    cut to about a millisecond) must end the kernel with a status bit, make later launches skip until the status
+    has been read, and leave the context usable."""
+    import torch
+    blocks = _pack([(256, 256, A.MOM_LOWRANK, 12, A.V_BLOCKMEAN, 1), (64, 64, A.MOM_FULL, 0, A.V_ELEMENT, 0)])
+    w = WL.Workload("expired", [], "bf16", "normal", steps=3)
+    run = ParityRun(w, True, lowrank_path=A.PATH_TENSOR, custom_blocks=blocks)
+    try:
+        run.step()
+        run.compare()
+        before = run.params.clone(), run.state.clone()
+        run.ctx.adapm_selftest_expired_wait()
+        # the status word is set: a step issued now must not write anything
+        run.ctx.adapm_step(run.params, run.grads, run.state, run.t + 1)
+        torch.cuda.synchronize()
+        assert torch.equal(before[0], run.params) and torch.equal(before[1], run.state)
+        assert run.ctx.adapm_get_status() == A.ST_WAIT_TEAM
+        assert run.ctx.adapm_get_status() == 0
+        run.step()                      # the same step number again, now for real: parity with the oracle holds
+        run.compare()
+    finally:
+        run.close()
 
 
 def test_tensor_path_nan_gradient_stays_in_its_block_and_does_not_hang():
@@ -336,3 +445,111 @@ def test_tensor_path_nan_gradient_stays_in_its_block_and_does_not_hang():
     assert np.isnan(p[:256 * 128]).any()
     assert np.isfinite(p[blocks[1].offset:]).all()           # the other block never sees it
     ctx.adapm_destroy()
+
+
+# ------------------------------------------------------------------------------------ ranks above 128, Llama3-8B shapes
+
+@pytest.mark.parametrize("rank", [160, 204])
+def test_tensor_path_ranks_above_128_20_steps(rank):
+    """Above rank 128 the refit takes the hi and the lo half of a factor in separate MMAs and the apply kernel
+    streams L as well as R; 20 steps against the oracle."""
+    blocks = _pack([(1536, 1024, A.MOM_LOWRANK, rank, A.V_BLOCKMEAN, 1),
+                    (640, 2048, A.MOM_LOWRANK, rank, A.V_ELEMENT, 0),
+                    (520, 392, A.MOM_LOWRANK, 24, A.V_BLOCKMEAN, 8)])      # a small rank beside them
+    w = WL.Workload("bigrank", [], "bf16", "normal", steps=20)
+    _run(w, True, 20, path=A.PATH_TENSOR, blocks=blocks, every=4)
+
+
+def test_llama3_8b_block_shapes_on_the_tensor_path():
+    """The four low-rank block shapes of the Llama3-8B-shaped set (Section 5.2: rank 5% of 4096 = 204, 51 for the
+    grouped-query key projection) at full size, and the whole set accepted by the tensor path: no block of it
+    falls back to the CUDA-core refit."""
+    w = WL.get_workload("llama3_8b")
+    blocks, _ = A.adapm_plan_default(w.tensors)
+    ctx = A.adapm_create(blocks, A.hparams(lowrank_path=A.PATH_TENSOR))       # would raise -6 otherwise
+    ctx.adapm_destroy()
+    shapes = sorted({(b.rows, b.cols, b.rank, b.v_group_rows) for b in blocks if b.mom_mode == A.MOM_LOWRANK})
+    assert shapes == [(1024, 4096, 51, 128), (4096, 4096, 204, 128), (4096, 14336, 204, 1), (14336, 4096, 204, 1)]
+    custom = _pack([(r, c, A.MOM_LOWRANK, k, A.V_BLOCKMEAN, g) for r, c, k, g in shapes])
+    _run(WL.Workload("llama3_shapes", [], "bf16", "normal", steps=3), True, 3, path=A.PATH_TENSOR, blocks=custom)
+
+
+@pytest.mark.parametrize("pct", [2, 10, 50])
+def test_rank_ratios_of_the_ablation(pct):
+    """Section 5.1.2 sweeps the rank over 2, 5, 10 and 50 percent of the full rank; at d = 1024 that is 20, 102 and
+    512.  Up to rank 256 the blocks run on the tensor path, above on the CUDA-core path (AUTO)."""
+    w = WL.get_workload("llama350m", rank_pct=pct)
+    blocks, _ = A.adapm_plan_default(w.tensors, rank_pct=pct)
+    sel = [i for i in sample_blocks(blocks, 1) if blocks[i].mom_mode == A.MOM_LOWRANK and blocks[i].rows <= 1024]
+    _run(w, True, 4, sel=sel, pooled=True, every=2)
+
+
+# ------------------------------------------------------------------------------------ global clipping, bf16 copy, finite check
+
+def _alternating(step):
+    return 0.5 if step % 2 else 2.0
+
+
+@pytest.mark.parametrize("path", [A.PATH_AUTO, A.PATH_SIMT])
+def test_llama60m_global_clipping_20_steps(path):
+    """Global gradient-norm clipping (Section 5.1, Setups).  The gradients of odd steps are halved and those of even
+    steps doubled, and the threshold sits between the two norms, so the clip factor is 1 on odd steps and below 1 on
+    even ones; the bf16 copy of the parameters is written along and must be the rounded fp32 parameters."""
+    import torch
+    w = WL.get_workload("llama60m")
+    blocks, _ = A.adapm_plan_default(w.tensors)
+    # ||g|| of this set is ~25 (sigma 1e-3, row scales log-uniform in [0.1, 10], 58 M elements)
+    run = ParityRun(w, True, oracle_blocks=sample_blocks(blocks, 1), lowrank_path=path, pooled_grads=True,
+                    hp_overrides=dict(max_grad_norm=25.0), grad_scale=_alternating, shadow=True)
+    seen = []
+    try:
+        for s in range(1, w.steps + 1):
+            run.step()
+            seen.append(run.last_gscale)
+            if s % 5 == 0 or s <= 2:
+                run.compare()
+                torch.cuda.synchronize()
+                assert torch.equal(run.shadow, run.params.to(torch.bfloat16))
+        assert run.ctx.adapm_get_status() == 0
+    finally:
+        run.close()
+    assert all(k == 1.0 for k in seen[0::2]) and all(0.3 < k < 0.9 for k in seen[1::2])
+
+
+def test_tiny_global_clipping_fp32_gradients():
+    w = WL.get_workload("tiny")
+    run = ParityRun(w, True, hp_overrides=dict(max_grad_norm=1.0), grad_scale=lambda s: 4.0 if s % 2 else 0.25,
+                    shadow=True)
+    try:
+        for _ in range(6):
+            run.step()
+            run.compare()
+        assert run.ctx.adapm_get_status() == 0
+        assert min(run.last_gscale, 1.0) <= 1.0
+    finally:
+        run.close()
+
+
+def test_finite_check_skips_the_step_and_reports_it():
+    """With ADAPM_FLAG_CHECK_FINITE a NaN or Inf anywhere in the gradients makes the whole step a no-op (parameters
+    and state untouched) and sets bit 64 of the status word; the next step with good gradients runs normally."""
+    import torch
+    blocks = _pack([(256, 128, A.MOM_LOWRANK, 8, A.V_BLOCKMEAN, 1), (64, 64, A.MOM_FULL, 0, A.V_ELEMENT, 0),
+                    (32, 64, A.MOM_NONE, 0, A.V_BLOCKMEAN, 1)])
+    w = WL.Workload("finite", [], "bf16", "normal", steps=3)
+    run = ParityRun(w, True, custom_blocks=blocks, hp_overrides=dict(flags=A.FLAG_CHECK_FINITE))
+    try:
+        run.step()
+        run.compare()
+        before = run.params.clone(), run.state.clone()
+        bad = run.grads.clone()
+        bad[blocks[1].offset + 5] = float("inf")
+        run.ctx.adapm_step(run.params, bad, run.state, run.t + 1)
+        torch.cuda.synchronize()
+        assert torch.equal(before[0], run.params) and torch.equal(before[1], run.state)
+        assert run.ctx.adapm_get_status() == A.ST_NONFINITE_GRAD
+        run.step()
+        run.compare()
+        assert run.ctx.adapm_get_status() == 0
+    finally:
+        run.close()

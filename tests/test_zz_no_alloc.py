@@ -10,6 +10,7 @@ import pytest
 
 import workloads as WL
 import paper_2510_09103_b200 as A
+from oracle import adapm_oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -17,7 +18,7 @@ pytestmark = pytest.mark.gpu
 def _device_grad(x, dtype):
     import torch
     vals, raw = WL.to_grad_dtype(x, dtype)
-    return torch.from_numpy(raw.view(np.int16) if dtype == "bf16" else raw).cuda()
+    return vals, torch.from_numpy(raw.view(np.int16) if dtype == "bf16" else raw).cuda()
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
@@ -28,7 +29,7 @@ def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row(dtype):
     # second call is smaller than the first, so it sees the first call's leftovers in the shared array
     shapes = [(37, 70001), (5, 4100)]
     for n_groups, ge in shapes:
-        g = _device_grad((rng.standard_normal(n_groups * ge) * 1e-3).astype(np.float32), dtype)
+        vals, g = _device_grad((rng.standard_normal(n_groups * ge) * 1e-3).astype(np.float32), dtype)
         want = torch.zeros(n_groups, device="cuda")
         scratch = torch.zeros(max(A.adapm_group_meansq_scratch_bytes(n_groups, ge) // 4, 64), device="cuda")
         A.adapm_group_meansq(g, gd, n_groups, ge, want, scratch)
@@ -38,6 +39,10 @@ def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row(dtype):
         w, h = want.cpu().numpy().astype(np.float64), got.cpu().numpy().astype(np.float64)
         assert np.isfinite(h).all() and (h > 0).all()
         assert np.abs(h - w).max() <= 1e-5 * np.abs(w).max()
+        # and against the definition itself: the group average of g^2 (the oracle's second moment from v = 0)
+        blk = O.Block(n_groups, ge, O.MOM_NONE, v_mode=O.V_BLOCKMEAN, v_group_rows=1)
+        ref = O.second_moment(np.zeros(n_groups), vals.astype(np.float64).reshape(n_groups, ge), blk, 0.0)
+        assert np.abs(h - ref).max() <= 1e-5 * np.abs(ref).max()
 
 
 def test_static_scratch_rejects_inputs_beyond_its_limit():

@@ -10,4 +10,4 @@ from .shapes import (  # noqa: F401
     ROLE_LM_HEAD, ROLE_VECTOR, ROLE_OTHER, Tensor, Workload, get_workload,
     WORKLOAD_NAMES,
 )
-from .gen import init_params, grad_for_tensor, to_grad_dtype, GradPool  # noqa: F401
+from .gen import init_params, grad_for_tensor, to_grad_dtype, GradPool, bf16_bits_to_f32, round_to_bf16_bits  # noqa: F401

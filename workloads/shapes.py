@@ -94,15 +94,17 @@ def _gpt2(n_layer: int, d: int, heads: int, ffn: int, vocab: int, ctx: int) -> L
     return t
 
 
-def _llama(n_layer: int, d: int, heads: int, ffn: int, vocab: int) -> List[Tensor]:
+def _llama(n_layer: int, d: int, heads: int, ffn: int, vocab: int, kv_heads: int = 0) -> List[Tensor]:
+    """kv_heads > 0: grouped-query attention, key and value projections have kv_heads * (d / heads) rows."""
+    kv_rows = d if kv_heads <= 0 else kv_heads * (d // heads)
     t: List[Tensor] = [Tensor("embed_tokens", ROLE_EMBED, vocab, d)]
     for i in range(n_layer):
         p = f"layers.{i}."
         t += [
             Tensor(p + "input_layernorm.weight", ROLE_VECTOR, 1, d, init="ones"),
             Tensor(p + "self_attn.q_proj", ROLE_Q, d, d, heads=heads),
-            Tensor(p + "self_attn.k_proj", ROLE_K, d, d, heads=heads),
-            Tensor(p + "self_attn.v_proj", ROLE_V, d, d),
+            Tensor(p + "self_attn.k_proj", ROLE_K, kv_rows, d, heads=heads if kv_heads <= 0 else kv_heads),
+            Tensor(p + "self_attn.v_proj", ROLE_V, kv_rows, d),
             Tensor(p + "self_attn.o_proj", ROLE_ATTN_OUT, d, d),
             Tensor(p + "post_attention_layernorm.weight", ROLE_VECTOR, 1, d, init="ones"),
             Tensor(p + "mlp.gate_proj", ROLE_MLP, ffn, d),
@@ -117,9 +119,10 @@ def _llama(n_layer: int, d: int, heads: int, ffn: int, vocab: int) -> List[Tenso
 
 
 WORKLOAD_NAMES = ("tiny", "llama60m", "gpt2_124m", "llama350m", "gpt2_1p5b")
+EXTRA_WORKLOAD_NAMES = ("llama3_8b",)      # Section 5.2's fine-tuning model, shapes only
 
 
-def get_workload(name: str, rank_override: int = 0) -> Workload:
+def get_workload(name: str, rank_override: int = 0, rank_pct: int = 5) -> Workload:
     """Return one of the five parameter sets.
 
     tiny       2-layer GPT-2 style, d=256, 4 heads, FFN 1024, vocab 4096, ctx 2048; fp32 grads.
@@ -127,16 +130,25 @@ def get_workload(name: str, rank_override: int = 0) -> Workload:
     gpt2_124m  12 layers, d=768, 12 heads, FFN 3072, vocab 50257, ctx 1024; bf16 Student-t grads.
     llama350m  24 layers, d=1024, 16 heads, SwiGLU 2736, vocab 32000; bf16 grads, 5% heavy rows.
     gpt2_1p5b  48 layers, d=1600, 25 heads, FFN 6400, vocab 50257, ctx 1024; bf16 Gaussian grads.
+    llama3_8b  32 layers, d=4096, 32 heads (8 key/value heads), SwiGLU 14336, vocab 128256, untied head; bf16
+               Gaussian grads.  The shapes of the model fine-tuned in Section 5.2; rank 5% of 4096 = 204.
+    "gpt2_1p5b@L" / "llama3_8b@L": the same shapes with L layers.  rank_pct: percent of the full rank (Section
+    5.1.2 sweeps 2, 5, 10 and 50).
     """
     layers = None
     if "@" in name:                  # "gpt2_1p5b@4": the same shapes with 4 layers (small profiling captures)
         name, _, n_l = name.partition("@")
         layers = int(n_l)
     if layers is not None:
-        if name != "gpt2_1p5b":
-            raise KeyError("a layer count can only be given for gpt2_1p5b")
-        w = Workload(f"{name}@{layers}", _gpt2(layers, 1600, 25, 6400, 50257, 1024), "bf16", "normal", steps=20)
+        if name == "gpt2_1p5b":
+            w = Workload(f"{name}@{layers}", _gpt2(layers, 1600, 25, 6400, 50257, 1024), "bf16", "normal", steps=20)
+        elif name == "llama3_8b":
+            w = Workload(f"{name}@{layers}", _llama(layers, 4096, 32, 14336, 128256, kv_heads=8), "bf16", "normal",
+                         steps=20)
+        else:
+            raise KeyError("a layer count can only be given for gpt2_1p5b and llama3_8b")
         w.rank_override = int(rank_override)
+        w.rank_pct = int(rank_pct)
         return w
     if name == "tiny":
         w = Workload(name, _gpt2(2, 256, 4, 1024, 4096, 2048), "f32", "normal", steps=10,
@@ -149,7 +161,10 @@ def get_workload(name: str, rank_override: int = 0) -> Workload:
         w = Workload(name, _llama(24, 1024, 16, 2736, 32000), "bf16", "heavyrows", steps=20)
     elif name == "gpt2_1p5b":
         w = Workload(name, _gpt2(48, 1600, 25, 6400, 50257, 1024), "bf16", "normal", steps=20)
+    elif name == "llama3_8b":
+        w = Workload(name, _llama(32, 4096, 32, 14336, 128256, kv_heads=8), "bf16", "normal", steps=20)
     else:
         raise KeyError(f"unknown workload {name!r}; choose from {WORKLOAD_NAMES}")
     w.rank_override = int(rank_override)
+    w.rank_pct = int(rank_pct)
     return w
