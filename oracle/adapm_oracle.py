@@ -33,6 +33,14 @@ Readings of the paper taken here (each is a choice; the paper does not settle it
     and nothing else changed.  Section 4.2's phrase "directly applying L_t R_t as the momentum" would instead
     give m^c := L_t R_t; the two differ by the residual r_t.  `correction=False` takes the first reading and
     `correction_off_uses_product=True` the second.
+  * "Update frequency T" (Section 5.1: T = 100; Section 5.1.2 sweeps it) is set but never defined: Algorithms 1
+    and 2 refit both factors at every step.  Reading taken for `refresh_period` = T > 1, PARITY UNPINNED (the
+    paper fixes nothing to check it against): the full refit of Algorithm 2 runs at steps 1, T+1, 2T+1, ...; at
+    the steps in between L is held and only R moves, by the R half of Algorithm 2 (same schedule, same K).
+    Everything else (lines 4, 6-9) is unchanged, so the correction of Eq. 3 still compensates the residual.
+    T = 1 is Algorithm 1 as printed.  The function itself is pinned to the mathematics (tests): T = 1 equals
+    the default, held-L passes equal scalar loops, and with orthonormal L and step size 1 one pass lands on
+    the least-squares R = L^T m_t.
 Parity with the authors' unreleased code on these readings is unpinned; what is
 pinned (tests/test_oracle_pins.py) is this oracle against closed forms, special
 cases, a library optimizer, the proof identity of Theorem 2 and brute force.
@@ -84,6 +92,7 @@ class HParams:
     correction: bool = True      # Eq. 3 on; off: m^c := m_t
     correction_off_uses_product: bool = False   # with correction off: m^c := L_t R_t instead of m_t
     max_grad_norm: float = math.inf   # global clipping threshold c; inf disables
+    refresh_period: int = 1      # T: both factors are refitted at steps 1, T+1, 2T+1, ...; in between only R
 
 
 @dataclass
@@ -105,8 +114,9 @@ def inner_schedule(K: int) -> List[float]:
 
 
 def lowrank_refit_gd(m_t: np.ndarray, L_prev: np.ndarray, R_prev: np.ndarray, K: int,
-                     scale: float = 1.0):
-    """Algorithm 2: warm start at (L_{t-1}, R_{t-1}); both derivatives from the same point."""
+                     scale: float = 1.0, update_L: bool = True):
+    """Algorithm 2: warm start at (L_{t-1}, R_{t-1}); both derivatives from the same point.
+    update_L=False holds L and moves only R (the steps between two refreshes, see `refresh_period`)."""
     L = np.array(L_prev, dtype=np.float64, copy=True)
     R = np.array(R_prev, dtype=np.float64, copy=True)
     if K <= 0:
@@ -115,7 +125,8 @@ def lowrank_refit_gd(m_t: np.ndarray, L_prev: np.ndarray, R_prev: np.ndarray, K:
         E = L @ R - m_t                  # L R - m_t
         dL = E @ R.T                     # dl/dL = (L R - m_t) R^T
         dR = L.T @ E                     # dl/dR = L^T (L R - m_t)
-        L = L - (scale * eta) * dL
+        if update_L:
+            L = L - (scale * eta) * dL
         R = R - (scale * eta) * dR
     return L, R
 
@@ -214,7 +225,8 @@ def block_step(W: np.ndarray, g: np.ndarray, st: BlockState, blk: Block, hp: HPa
         P_prev = st.L @ st.R
         m_t = (1.0 - b1) * g + b1 * P_prev                     # line 4
         if solver == "gd":
-            L, R = lowrank_refit_gd(m_t, st.L, st.R, hp.inner_iters, hp.inner_lr_scale)   # line 5
+            refresh = hp.refresh_period <= 1 or (t - 1) % hp.refresh_period == 0
+            L, R = lowrank_refit_gd(m_t, st.L, st.R, hp.inner_iters, hp.inner_lr_scale, update_L=refresh)   # line 5
         elif solver == "exact":
             L, R = lowrank_refit_exact(m_t, blk.rank)
         else:

@@ -514,3 +514,57 @@ def test_inner_lr_scale_multiplies_every_step_size():
     np.testing.assert_allclose(R[0], r, rtol=1e-13)
     L2, R2 = O.lowrank_refit_gd(tgt, L0, R0, 5, 0.0)
     assert np.array_equal(L2, L0) and np.array_equal(R2, R0)
+
+
+# ------------------------------------------------------------------------------------ refresh period T
+
+def test_refresh_period_one_is_algorithm_1_as_printed():
+    blk = O.Block(8, 6, O.MOM_LOWRANK, rank=2, weight_decay=0.1)
+    L0 = O.init_L0(8, 2, 0, 0)
+    a, b = O.new_state(blk, L0), O.new_state(blk, L0)
+    Wa = RNG.standard_normal((8, 6)); Wb = Wa.copy()
+    for t in range(1, 7):
+        g = RNG.standard_normal((8, 6)) * 1e-2
+        Wa = O.block_step(Wa, g, a, blk, O.HParams(), t)
+        Wb = O.block_step(Wb, g, b, blk, O.HParams(refresh_period=1), t)
+        assert np.array_equal(Wa, Wb) and np.array_equal(a.L, b.L) and np.array_equal(a.R, b.R)
+
+
+def test_refresh_period_holds_L_between_refreshes_and_moves_R():
+    T = 3
+    blk = O.Block(8, 6, O.MOM_LOWRANK, rank=2)
+    st = O.new_state(blk, O.init_L0(8, 2, 0, 0))
+    W = RNG.standard_normal((8, 6))
+    for t in range(1, 9):
+        L_before, R_before = st.L.copy(), st.R.copy()
+        W = O.block_step(W, RNG.standard_normal((8, 6)) * 1e-2, st, blk, O.HParams(refresh_period=T), t, keep=True)
+        if (t - 1) % T == 0:
+            assert not np.array_equal(st.L, L_before)
+        else:
+            assert np.array_equal(st.L, L_before)
+        assert not np.array_equal(st.R, R_before)
+        # lines 6 and 8 are unchanged: the corrected momentum is g + c (P_{t-1} - P_t) whatever the solver did
+        c = 0.9 / (1 - 0.9)
+        np.testing.assert_allclose(st.last["m_c"], (st.last["m_t"] - 0.9 * st.last["P_prev"]) / 0.1
+                                   + c * (st.last["P_prev"] - st.last["P"]), rtol=1e-10, atol=1e-15)
+
+
+def test_held_L_passes_equal_scalar_loops_and_hit_least_squares_with_orthonormal_L():
+    m, n = 3, 2
+    tgt = RNG.standard_normal((m, n))
+    L0 = RNG.standard_normal((m, 1)); R0 = RNG.standard_normal((1, n))
+    L, R = O.lowrank_refit_gd(tgt, L0, R0, 5, 1.0, update_L=False)
+    l = [float(x) for x in L0[:, 0]]; r = [float(x) for x in R0[0]]
+    for k in range(1, 6):
+        eta = 0.5 * (1.0 + math.cos(math.pi * k / 5))
+        dr = [sum(l[i] * (l[i] * r[j] - tgt[i, j]) for i in range(m)) for j in range(n)]
+        r = [r[j] - eta * dr[j] for j in range(n)]
+    assert np.array_equal(L, L0)
+    np.testing.assert_allclose(R[0], r, rtol=1e-13)
+    # orthonormal L, one pass with step size exactly 1 (K = 1 would give eta_1 = 0, so use K = 2 scaled to eta_1 = 1):
+    # R_1 = R_0 - (L^T L R_0 - L^T m) = L^T m, the least-squares solution for that L
+    Q = np.linalg.qr(RNG.standard_normal((7, 3)))[0]
+    tgt = RNG.standard_normal((7, 5))
+    eta1 = 0.5 * (1.0 + math.cos(math.pi / 2))
+    _, R1 = O.lowrank_refit_gd(tgt, Q, RNG.standard_normal((3, 5)), 2, 1.0 / eta1, update_L=False)
+    np.testing.assert_allclose(R1, Q.T @ tgt, rtol=1e-12, atol=1e-14)
