@@ -398,7 +398,8 @@ def run_gpu(args) -> None:
     flags = ((A.FLAG_NO_PANEL_TEAMS if args.teams == "off" else 0) | (A.FLAG_FORCE_PANEL_TEAMS if args.teams == "force" else 0)
              | (A.FLAG_NO_SUMSQ_FOLD if args.no_fold else 0))
     hp = A.hparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, grad_dtype=gd, lowrank_path=path, flags=flags,
-                   tune_panels=args.panels, tune_stage_k=args.stage_k)
+                   tune_panels=args.panels, tune_stage_k=args.stage_k, max_grad_norm=args.max_grad_norm,
+                   refresh_period=args.refresh_period)
     ctx = A.adapm_create(blocks, hp)
 
     # synthetic inputs: parameters N(0, 0.02^2) drawn on the device; gradients tiled from a seeded host pool
@@ -408,11 +409,28 @@ def run_gpu(args) -> None:
     raw = pool.raw.view(np.int16) if w.grad_dtype == "bf16" else pool.raw
     tdt = torch.int16 if w.grad_dtype == "bf16" else torch.float32
     pool_t = torch.from_numpy(raw)
-    grads_host = torch.empty(total, dtype=tdt, pin_memory=True)
-    reps = -(-total // pool_t.numel())
-    grads_host.copy_(pool_t.repeat(reps)[:total])
+    # sets beyond 2e9 parameters: no end-to-end leg (48+ GB of pinned host memory) and the gradients are tiled on
+    # the device
+    if total > 2_000_000_000:
+        args.no_e2e = True
     grads = torch.empty(total, dtype=torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32, device=dev)
-    grads.view(tdt).copy_(grads_host)
+    grads_host = None
+    if args.no_e2e:
+        pool_d = pool_t.to(dev)
+        gv = grads.view(tdt)
+        for i in range(0, total, pool_d.numel()):
+            n = min(pool_d.numel(), total - i)
+            gv[i:i + n].copy_(pool_d[:n])
+        del pool_d
+    else:
+        grads_host = torch.empty(total, dtype=tdt, pin_memory=True)
+        reps = -(-total // pool_t.numel())
+        grads_host.copy_(pool_t.repeat(reps)[:total])
+        grads.view(tdt).copy_(grads_host)
+    shadow = None
+    if args.shadow:
+        shadow = torch.zeros(total, dtype=torch.bfloat16, device=dev)
+        ctx.adapm_set_shadow_params(shadow)
     state = torch.zeros(ctx.adapm_state_bytes() // 4, dtype=torch.float32, device=dev)
     work = torch.zeros(max(ctx.adapm_workspace_bytes() // 4, 64), dtype=torch.float32, device=dev)
     ctx.adapm_set_workspace(work)
@@ -513,6 +531,7 @@ def run_gpu(args) -> None:
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "params": w.numel, "blocks": len(blocks), "v_mode": args.v_mode,
+                   "max_grad_norm": args.max_grad_norm, "refresh_period": args.refresh_period, "bf16_shadow": args.shadow,
                    "grad_dtype": w.grad_dtype, "state_dtype": "f32", "lowrank_path": args.path,
                    "lowrank_kernels": "tensor" if any(k.startswith("tc_") for k in kernels) else "simt",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
@@ -558,6 +577,9 @@ def main() -> None:
     ap.add_argument("--stage-k", type=int, default=0, help="tensor path: K per stage, 64 or 128 (0 = automatic)")
     ap.add_argument("--teams", default="auto", choices=["auto", "off", "force"], help="panel team schedule")
     ap.add_argument("--no-fold", action="store_true", help="row sums of g^2 from a pass of their own")
+    ap.add_argument("--max-grad-norm", type=float, default=0.0, help="global gradient-norm clipping threshold (0 = off)")
+    ap.add_argument("--refresh-period", type=int, default=0, help="T: refit both factors every T steps (0/1 = every step)")
+    ap.add_argument("--shadow", action="store_true", help="also write the bf16 copy of the parameters")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -110,6 +110,10 @@ typedef struct {
   uint32_t flags;          /* ADAPM_FLAG_*; 0 = defaults                                           */
   float   max_grad_norm;   /* global gradient clipping (Section 5.1: threshold 1.0): every gradient is
                               multiplied by min(1, c / ||g||_2), the norm over all blocks; 0 or +inf = off */
+  int32_t refresh_period;  /* T of Section 5.1 ("update frequency"; the paper sets 100 and does not define
+                              it).  Reading: both factors are refitted by Algorithm 2 at steps 1, T+1,
+                              2T+1, ...; in between L is held and only R moves (the R half of Algorithm 2).
+                              0 or 1 = Algorithm 1 as printed, every step                          */
   int32_t tune_panels;     /* tensor path: 128-row panels per refit item (1..3); 0 = automatic     */
   int32_t tune_stage_k;    /* tensor path: K per shared-memory stage (64 or 128); 0 = automatic    */
 } adapm_hparams;
@@ -194,7 +198,7 @@ int64_t adapm_launch_count(const adapm_ctx* ctx);
 
 /*
  * Measurement aid: with profiling on, adapm_step records a CUDA event on `stream` before its first
- * and after each of its kernels.  adapm_get_launch_times waits for the last step's events and
+ * and after each of its kernels, and wraps each launch in an NVTX range named after its kind.  adapm_get_launch_times waits for the last step's events and
  * returns each kernel's duration in milliseconds and its kind (see adapm_launch_kind_name);
  * with ms == kinds == NULL it only reports the number of launches.
  */

@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [
         _nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
         "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-        "-o", LIB_PATH,
+        "-o", LIB_PATH, "-ldl",
     ]
     if verbose:
         cmd += ["-Xptxas", "-v"]

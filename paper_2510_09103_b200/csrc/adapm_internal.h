@@ -134,7 +134,8 @@ enum LaunchKind : int32_t {
   LK_REDUCE_PARTIAL, LK_REDUCE_FINAL, LK_STREAM, LK_GEMM, LK_APPLY_SIMT, LK_COMMIT,
   LK_TC_CONVERT, LK_TC_GRAM, LK_TC_PANEL, LK_TC_APPLY,
   LK_REDUCE_ROWS,       // reduce_final over the row sums of g^2 that the first refit pass left
-  LK_GRADNORM           // global gradient norm and the clip factor
+  LK_GRADNORM,          // global gradient norm and the clip factor
+  LK_TC_COPY            // previous split copy of L -> final set (steps that hold L)
 };
 // when a launch of the program runs
 enum LaunchWhen : int32_t {
@@ -149,6 +150,7 @@ struct Launch {
   int64_t aux0 = 0, aux1 = 0, aux2 = 0, aux3 = 0, aux4 = 0, aux5 = 0;
   int32_t when = WHEN_ALWAYS;
   int32_t only_convert = 0;   // 1: only in a step that rebuilds the split copies of the factors
+  int32_t phase = 0;          // 0: every step; 1: only steps that refit both factors; 2: only steps that hold L
 };
 
 // ---------------------------------------------------------------------------------------------

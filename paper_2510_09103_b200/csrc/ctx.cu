@@ -6,6 +6,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "adapm_internal.h"
 
 namespace adapm {
@@ -36,6 +38,7 @@ int validate(const adapm_block* blocks, int64_t n, const adapm_hparams& hp) {
   if (!std::isfinite(hp.lr) || !std::isfinite(hp.inner_lr_scale)) return ADAPM_EINVAL;
   if (hp.grad_dtype != ADAPM_GRAD_F32 && hp.grad_dtype != ADAPM_GRAD_BF16) return ADAPM_EINVAL;
   if (hp.lowrank_path < ADAPM_PATH_AUTO || hp.lowrank_path > ADAPM_PATH_TENSOR) return ADAPM_EINVAL;
+  if (hp.refresh_period < 0) return ADAPM_ERANGE;
   if (!(hp.max_grad_norm >= 0.f)) return ADAPM_ERANGE;      // 0 and +inf both mean "no clipping"; NaN is refused
   if (hp.tune_panels < 0 || hp.tune_panels > 3) return ADAPM_ERANGE;
   if (hp.tune_stage_k != 0 && hp.tune_stage_k != 64 && hp.tune_stage_k != 128) return ADAPM_ERANGE;
@@ -160,9 +163,15 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
 
   // ---- streaming blocks and reduction jobs -------------------------------------------------------
   std::vector<StreamBlk> sblk;
-  std::vector<ReduceJob> rjobs;
-  int64_t cta_cursor = 0, work_cursor = 0, unit_cursor = 0, group_cursor = 0;
-  auto add_reduce_job = [&](int i, int64_t group_elems, int64_t n_groups) {
+  // two-stage group sums of g^2: `rjobs` run every step, `rjobs_hold` only in steps that hold L (there the
+  // tensor path has no row panels to take the row sums from)
+  struct ReduceSet { std::vector<ReduceJob> jobs; int64_t units = 0, groups = 0; };
+  ReduceSet rset_all, rset_hold;
+  int64_t cta_cursor = 0, work_cursor = 0;
+  auto add_reduce_job = [&](ReduceSet& rs, int i, int64_t group_elems, int64_t n_groups) {
+    std::vector<ReduceJob>& rjobs = rs.jobs;
+    int64_t& unit_cursor = rs.units;
+    int64_t& group_cursor = rs.groups;
     ReduceJob j;
     std::memset(&j, 0, sizeof(j));
     j.g_off = c->blocks[i].offset;
@@ -199,7 +208,7 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
       s.units_per_group = (int32_t)((group_elems + kWarpUnitMax - 1) / kWarpUnitMax);
       s.n_units = n_groups * s.units_per_group;
       s.vec_ok = (group_elems % kChunkElems == 0 || n_groups == 1) ? 1 : 0;
-      add_reduce_job(i, group_elems, n_groups);
+      add_reduce_job(rset_all, i, group_elems, n_groups);
     }
     s.first_cta = cta_cursor;
     cta_cursor += s.team == 32 ? (s.n_units + 7) / 8 : s.n_units;
@@ -209,14 +218,15 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   // Group sums of g^2 of the low-rank blocks come from the reduction kernels, except on the tensor path when
   // there is a refit pass: its row panels read every row of g anyway and leave the row sums behind.
   const bool fold_sumsq = K_eff > 0 && !(hp->flags & ADAPM_FLAG_NO_SUMSQ_FOLD);
+  const bool with_hold = hp->refresh_period > 1 && K_eff > 0;
   for (int pass = 0; pass < 2; ++pass) {
-    if (pass == 1 && fold_sumsq) break;
+    if (pass == 1 && fold_sumsq && !with_hold) break;
     for (int64_t i : (pass == 0 ? lowrank_ids : tc_ids)) {
       const adapm_block& b = c->blocks[i];
       if (b.v_mode != ADAPM_V_BLOCKMEAN) continue;
       const int64_t numel = (int64_t)b.rows * b.cols;
       const int64_t group_elems = b.v_group_rows == 0 ? numel : (int64_t)b.v_group_rows * b.cols;
-      add_reduce_job((int)i, group_elems, numel / group_elems);
+      add_reduce_job((pass == 1 && fold_sumsq) ? rset_hold : rset_all, (int)i, group_elems, numel / group_elems);
     }
   }
 
@@ -240,19 +250,25 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     prog.push_back(GN);
     c->use_gscale = 1;
   }
-  if (!rjobs.empty()) {
+  for (int which = 0; which < 2; ++which) {
+    const ReduceSet& rs = which ? rset_hold : rset_all;
+    const std::vector<ReduceJob>& rjobs = rs.jobs;
+    if (rjobs.empty()) continue;
     const int64_t off = append_table(c->h_tables, rjobs);
     // CTA index -> job of the CTA's first unit (the job table is sorted by first_unit), so that a warp finds its job
     // with a step or two instead of a binary search
-    std::vector<int32_t> cta_job((size_t)((unit_cursor + 7) / 8));
+    std::vector<int32_t> cta_job((size_t)((rs.units + 7) / 8));
     for (size_t q = 0, j = 0; q < cta_job.size(); ++q) {
       while (j + 1 < rjobs.size() && rjobs[j + 1].first_unit <= (int64_t)q * 8) ++j;
       cta_job[q] = (int32_t)j;
     }
-    Launch RP{LK_REDUCE_PARTIAL, off, (int64_t)rjobs.size(), (unit_cursor + 7) / 8, unit_cursor};
+    Launch RP{LK_REDUCE_PARTIAL, off, (int64_t)rjobs.size(), (rs.units + 7) / 8, rs.units};
     RP.aux1 = append_table(c->h_tables, cta_job);
+    RP.phase = which ? 2 : 0;
     prog.push_back(RP);
-    prog.push_back({LK_REDUCE_FINAL, off, (int64_t)rjobs.size(), (group_cursor + 7) / 8, group_cursor});
+    Launch RF{LK_REDUCE_FINAL, off, (int64_t)rjobs.size(), (rs.groups + 7) / 8, rs.groups};
+    RF.phase = RP.phase;
+    prog.push_back(RF);
   }
   if (!sblk.empty()) {
     const int64_t off = append_table(c->h_tables, sblk);
@@ -301,6 +317,10 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     const float b1 = hp->beta1, a1 = 1.f - hp->beta1;
     int src_base = BASE_STATE; int64_t src_shift = 0;   // where the current iterate lives
     int dst_buf = 0;
+    // with a refresh period the passes exist twice: refitting both factors (phase 1) and holding L (phase 2)
+    for (int phase = (with_hold ? 1 : 0); phase <= (with_hold ? 2 : 0); ++phase) {
+    const bool hold = phase == 2;
+    src_base = BASE_STATE; src_shift = 0; dst_buf = 0;
     for (int it = 0; it < K_eff; ++it) {
       const float se = (float)etas[it];
       const int64_t dst_shift = c->ws_lr[dst_buf];
@@ -329,7 +349,7 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         // A = g R^T  (m x r), contraction over n
         reset(); p.x_base = BASE_GRADS; p.x_off = b.offset; p.sxi = nn; p.sxk = 1;
         p.y_base = (int8_t)src_base; p.y_off = Rc; p.syk = 1; p.syj = nn;
-        p.c_base = BASE_WORK; p.c_off = Aw; p.M = m; p.N = r; p.K = nn; p.ldc = r; push(pAB, p, tAB);
+        p.c_base = BASE_WORK; p.c_off = Aw; p.M = m; p.N = r; p.K = nn; p.ldc = r; if (!hold) push(pAB, p, tAB);
         // B = L^T g  (r x n), contraction over m
         reset(); p.x_base = (int8_t)src_base; p.x_off = Lc; p.sxi = 1; p.sxk = r;
         p.y_base = BASE_GRADS; p.y_off = b.offset; p.syk = nn; p.syj = 1;
@@ -337,8 +357,8 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         // G1 = R R^T, G2 = R0 R^T  (contraction over n)
         reset(); p.x_base = (int8_t)src_base; p.x_off = Rc; p.sxi = nn; p.sxk = 1;
         p.y_base = (int8_t)src_base; p.y_off = Rc; p.syk = 1; p.syj = nn;
-        p.c_base = BASE_WORK; p.c_off = G1; p.M = r; p.N = r; p.K = nn; p.ldc = r; push(pG, p, tG);
-        p.x_base = BASE_STATE; p.x_off = R0; p.c_off = G2; push(pG, p, tG);
+        p.c_base = BASE_WORK; p.c_off = G1; p.M = r; p.N = r; p.K = nn; p.ldc = r; if (!hold) push(pG, p, tG);
+        p.x_base = BASE_STATE; p.x_off = R0; p.c_off = G2; if (!hold) push(pG, p, tG);
         // G3 = L^T L, G4 = L^T L0  (contraction over m)
         reset(); p.x_base = (int8_t)src_base; p.x_off = Lc; p.sxi = 1; p.sxk = r;
         p.y_base = (int8_t)src_base; p.y_off = Lc; p.syk = r; p.syj = 1;
@@ -349,11 +369,13 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         p.y_base = BASE_WORK; p.y_off = G1; p.syk = r; p.syj = 1;
         p.c_base = BASE_WORK; p.c_off = Ld; p.M = m; p.N = r; p.K = r; p.ldc = r;
         p.alpha = -se; p.beta = 0.f; p.z1_base = (int8_t)src_base; p.z1_off = Lc; p.c1 = 1.f;
-        p.z2_base = BASE_WORK; p.z2_off = Aw; p.c2 = se * a1; push(pU1, p, tU1);
+        p.z2_base = BASE_WORK; p.z2_off = Aw; p.c2 = se * a1;
+        if (hold) { p.K = 0; p.alpha = 0.f; p.z2_base = BASE_NONE; p.c2 = 0.f; }      // L' = L
+        push(pU1, p, tU1);
         reset(); p.x_base = BASE_STATE; p.x_off = L0; p.sxi = r; p.sxk = 1;
         p.y_base = BASE_WORK; p.y_off = G2; p.syk = r; p.syj = 1;
         p.c_base = BASE_WORK; p.c_off = Ld; p.M = m; p.N = r; p.K = r; p.ldc = r;
-        p.alpha = se * b1; p.beta = 1.f; push(pU2, p, tU2);
+        p.alpha = se * b1; p.beta = 1.f; if (!hold) push(pU2, p, tU2);
         // R' = R - se ( G3 R - b1 G4 R0 - a1 B )
         reset(); p.x_base = BASE_WORK; p.x_off = G3; p.sxi = r; p.sxk = 1;
         p.y_base = (int8_t)src_base; p.y_off = Rc; p.syk = nn; p.syj = 1;
@@ -365,13 +387,16 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         p.c_base = BASE_WORK; p.c_off = Rd; p.M = r; p.N = nn; p.K = r; p.ldc = nn;
         p.alpha = se * b1; p.beta = 1.f; push(pU2, p, tU2);
       }
-      prog.push_back({LK_GEMM, append_table(c->h_tables, pAB), (int64_t)pAB.size(), tAB});
-      prog.push_back({LK_GEMM, append_table(c->h_tables, pG), (int64_t)pG.size(), tG});
-      prog.push_back({LK_GEMM, append_table(c->h_tables, pU1), (int64_t)pU1.size(), tU1});
-      prog.push_back({LK_GEMM, append_table(c->h_tables, pU2), (int64_t)pU2.size(), tU2});
+      for (auto* pv : {&pAB, &pG, &pU1, &pU2}) {
+        const int64_t tiles = pv == &pAB ? tAB : (pv == &pG ? tG : (pv == &pU1 ? tU1 : tU2));
+        Launch GL{LK_GEMM, append_table(c->h_tables, *pv), (int64_t)pv->size(), tiles};
+        GL.phase = phase;
+        prog.push_back(GL);
+      }
       src_base = BASE_WORK; src_shift = dst_shift;
       c->final_lr_buf = dst_buf;
       dst_buf ^= 1;
+    }
     }
     // apply
     std::vector<ApplyBlk> ab;
@@ -498,7 +523,7 @@ extern "C" int64_t adapm_launch_count(const adapm_ctx* c) {
   if (c->last_step_launches > 0) return c->last_step_launches;
   int64_t n = 0;
   for (const Launch& L : c->program)
-    if ((L.when == WHEN_ALWAYS || L.when == WHEN_EVEN) && !L.only_convert) ++n;
+    if ((L.when == WHEN_ALWAYS || L.when == WHEN_EVEN) && !L.only_convert && L.phase != 2) ++n;
   return n;
 }
 
@@ -548,6 +573,8 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
   b.status = c->d_status; b.gscale = c->d_gscale; b.shadow = (uint16_t*)c->shadow;
   float* work = (float*)c->workspace;
 
+  // refresh period T: both factors are refitted at steps 1, T+1, 2T+1, ...; the steps in between hold L
+  const bool refresh = hp.refresh_period <= 1 || (t - 1) % hp.refresh_period == 0;
   int parity = 0, convert = 0;
   if (c->tc) {
     const int prc = tensor_prepare_step(c, b, t, s, &parity, &convert);
@@ -560,10 +587,12 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
   }
   size_t li = 0;
   for (const Launch& L : c->program) {
-    if ((L.only_convert && !convert) || (L.when == WHEN_EVEN && parity != 0) || (L.when == WHEN_ODD && parity != 1))
+    if ((L.only_convert && !convert) || (L.when == WHEN_EVEN && parity != 0) || (L.when == WHEN_ODD && parity != 1) ||
+        (L.phase == 1 && !refresh) || (L.phase == 2 && refresh))
       continue;
     const unsigned char* tab = c->d_tables + L.table_off;
     int rc = ADAPM_OK;
+    if (prof) nvtxRangePushA(adapm_launch_kind_name((int32_t)L.kind));   // a named range per launch for timeline tools
     switch (L.kind) {
       case LK_GRADNORM:
         rc = launch_gradnorm((const NormRange*)tab, (const int32_t*)(c->d_tables + L.aux0), L.grid, grads, hp.grad_dtype,
@@ -591,6 +620,7 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
       default:
         rc = run_tensor_launch(c, L, b, sc, parity, s); break;
     }
+    if (prof) nvtxRangePop();
     if (rc != ADAPM_OK) return rc;
     ++li;
     if (prof) {
@@ -636,6 +666,7 @@ extern "C" const char* adapm_launch_kind_name(int32_t kind) {
     case LK_REDUCE_FINAL: return "reduce_final";
     case LK_REDUCE_ROWS: return "reduce_rows";
     case LK_GRADNORM: return "grad_norm";
+    case LK_TC_COPY: return "tc_copy";
     case LK_STREAM: return "stream_update";
     case LK_GEMM: return "gemm_simt";
     case LK_APPLY_SIMT: return "apply_simt";

@@ -95,6 +95,31 @@ __global__ void __launch_bounds__(256) tc_convert_kernel(const ConvertJob* __res
   }
 }
 
+struct CopyJob {
+  int64_t src_off, dst_off;   // bf16 element offsets in the workspace
+  int32_t rows, width;        // width in elements (a multiple of 8)
+  int32_t src_ld, dst_ld;
+  int64_t first_row;          // prefix sum of rows
+};
+
+// rows of `width` bf16 from one split array to another (a step that holds L carries its split copy over)
+__global__ void __launch_bounds__(256) tc_copy_kernel(const CopyJob* __restrict__ jobs, int n_jobs, int64_t total_rows,
+                                                      uint16_t* __restrict__ work, const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= total_rows) return;
+  int lo = 0, hi = n_jobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (jobs[mid].first_row <= row) lo = mid; else hi = mid - 1;
+  }
+  const CopyJob J = jobs[lo];
+  const int64_t r = row - J.first_row;
+  const uint4* src = reinterpret_cast<const uint4*>(work + J.src_off + r * J.src_ld);
+  uint4* dst = reinterpret_cast<uint4*>(work + J.dst_off + r * J.dst_ld);
+  for (int i = threadIdx.x & 31; i < J.width / 8; i += 32) dst[i] = src[i];
+}
+
 }  // namespace
 
 // Host side of the tensor path, owned by the context.
@@ -416,10 +441,29 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     prog.push_back(L);
   }
 
-  // ---- refit passes, once per parity of the step -----------------------------------------------------------
+  // ---- refit passes, once per parity of the step and per kind of step ------------------------------------------
+  // With a refresh period T > 1 a step either refits both factors (phase 1) or holds L and refits R (phase 2:
+  // Gram matrices of L only, column panels only, and the split copy of L carried over to the final set).
   const int team_mode = (hp.flags & ADAPM_FLAG_NO_PANEL_TEAMS) ? 1 : ((hp.flags & ADAPM_FLAG_FORCE_PANEL_TEAMS) ? 2 : 0);
-  for (int parity = 0; parity < (P->rotate ? 2 : 1); ++parity) {
+  const bool with_hold = hp.refresh_period > 1 && K_eff > 0;
+  for (int parity = 0; parity < (P->rotate ? 2 : 1); ++parity)
+  for (int phase = (with_hold ? 1 : 0); phase <= (with_hold ? 2 : 0); ++phase) {
+    const bool hold = phase == 2;
     const int prev = parity, fin = 1 - parity;
+    const int when = P->rotate ? (parity ? WHEN_ODD : WHEN_EVEN) : WHEN_ALWAYS;
+    if (hold) {
+      std::vector<CopyJob> jobs;
+      int64_t rows = 0;
+      for (const TcBlock& t : P->blk) {
+        const adapm_block& b = c->blocks[t.id];
+        CopyJob j{t.lc[prev], t.lc[fin], b.rows, 2 * t.half, t.ld[prev], t.ld[fin], rows};
+        rows += b.rows;
+        jobs.push_back(j);
+      }
+      Launch CP{LK_TC_COPY, append_items(c->h_tables, jobs), (int64_t)jobs.size(), (rows + 7) / 8};
+      CP.aux0 = rows; CP.when = when; CP.phase = phase;
+      prog.push_back(CP);
+    }
     int src = prev;
     for (int pass = 0; pass < K_eff; ++pass) {
       const int dst = ((K_eff - 1 - pass) % 2 == 0) ? fin : 2;
@@ -459,10 +503,13 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
             grams.push_back(it);
           }
         };
-        gram(mb + MAP_RTCT + src, mb + MAP_RTCN + src, n, 0, -1.f / a1);    // Bop1[j][k] = -(R R^T)[j][k] / (1-b1), stored as [k][j]
-        gram(mb + MAP_RTCT + prev, mb + MAP_RTCN + src, n, 1, b1 / a1);     // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
-        gram(mb + MAP_LCT + src, mb + MAP_LCN + src, m, 2, -1.f / a1);      // Bop3[j][k] = -(L^T L)[j][k] / (1-b1)
-        gram(mb + MAP_LCT + prev, mb + MAP_LCN + src, m, 3, b1 / a1);       // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
+        const int srcL = hold ? prev : src;     // a held L stays in the previous set all step long
+        if (!hold) {
+          gram(mb + MAP_RTCT + src, mb + MAP_RTCN + src, n, 0, -1.f / a1);  // Bop1[j][k] = -(R R^T)[j][k] / (1-b1), stored as [k][j]
+          gram(mb + MAP_RTCT + prev, mb + MAP_RTCN + src, n, 1, b1 / a1);   // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
+        }
+        gram(mb + MAP_LCT + srcL, mb + MAP_LCN + srcL, m, 2, -1.f / a1);    // Bop3[j][k] = -(L^T L)[j][k] / (1-b1)
+        gram(mb + MAP_LCT + prev, mb + MAP_LCN + srcL, m, 3, b1 / a1);      // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
 
         // one item = up to n_pan adjacent panels of 128 owners that share every B box
         auto panel = [&](bool is_L, int p0, int np) {
@@ -471,7 +518,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           const int mS = (is_L ? mb + MAP_LC : mb + MAP_RTC) + src, m0 = (is_L ? mb + MAP_LC : mb + MAP_RTC) + prev;
           const int g1 = mb + MAP_GS + (is_L ? 0 : 2), g2 = g1 + 1;
           if (is_L) it.seg[0] = make_seg(geo, mb + MAP_G, 0, p0, 0, np, 0, 128, mb + MAP_RTCN + src, rp, half, n, 0, 2 * rp, 1);  // g R^T
-          else it.seg[0] = make_seg(geo, mb + MAP_GT, p0, 0, 1, np, 128, 0, mb + MAP_LCN + src, rp, half, m, 0, 2 * rp, 1);       // g^T L
+          else it.seg[0] = make_seg(geo, mb + MAP_GT, p0, 0, 1, np, 128, 0, mb + MAP_LCN + srcL, rp, half, m, 0, 2 * rp, 1);      // g^T L
           // [hi | lo] of the current and of the previous factor against the stacked Gram operands
           it.seg[1] = make_seg(geo, mS, 0, p0, 0, np, 0, 128, g1, rp, half, half + rp, 0, 2 * rp, 0);
           it.seg[2] = make_seg(geo, m0, 0, p0, 0, np, 0, 128, g2, rp, half, half + rp, 0, 2 * rp, 0);
@@ -488,7 +535,8 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
         };
         BlockSpan sp;
         sp.first = panels.size();
-        for (int p0 = 0; p0 < m; p0 += 128 * n_pan) panel(true, p0, std::min(n_pan, (m - p0 + 127) / 128));
+        if (!hold)
+          for (int p0 = 0; p0 < m; p0 += 128 * n_pan) panel(true, p0, std::min(n_pan, (m - p0 + 127) / 128));
         sp.n_row = panels.size() - sp.first;
         for (int p0 = 0; p0 < n; p0 += 128 * n_pan) panel(false, p0, std::min(n_pan, (n - p0 + 127) / 128));
         sp.n_col = panels.size() - sp.first - sp.n_row;
@@ -504,7 +552,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       G.aux1 = 2 * G.aux0 <= 512 ? 2 : 1; G.aux2 = gram_na;
       G.aux3 = append_items(c->h_tables, begin_g);
       G.aux4 = -1; G.aux5 = 0;
-      G.when = P->rotate ? (parity ? WHEN_ODD : WHEN_EVEN) : WHEN_ALWAYS;
+      G.when = when; G.phase = phase;
       prog.push_back(G);
       Launch Q{LK_TC_PANEL, append_items(c->h_tables, panels), (int64_t)panels.size(), grid_p};
       Q.aux0 = n_pan * 2 * rp_max; Q.aux1 = 2 * Q.aux0 <= 512 ? 2 : 1;
@@ -513,11 +561,11 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       // one accumulator buffer that leaves room to park the sums D0 + D1 of its panels (rp columns each)
       Q.aux4 = (Q.aux1 == 1 && Q.aux0 + n_pan * rp_max <= 512) ? Q.aux0 : -1;
       Q.aux5 = any_sumsq ? 1 : 0;
-      Q.when = G.when;
+      Q.when = when; Q.phase = phase;
       prog.push_back(Q);
-      if (pass == 0 && !row_jobs.empty()) {
+      if (pass == 0 && !row_jobs.empty() && !hold) {
         Launch RF{LK_REDUCE_ROWS, 0, 0, 0};       // table filled in by the caller (shared by both parities)
-        RF.when = G.when;
+        RF.when = when; RF.phase = phase;
         prog.push_back(RF);
       }
       src = dst;
@@ -705,6 +753,10 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       tc_convert_kernel<<<(unsigned)L.grid, 256, 0, s>>>((const ConvertJob*)tab, (int)L.n_items, L.aux0,
                                                         (const float*)b.p[BASE_STATE], (uint16_t*)b.p[BASE_WORK],
                                                         c->d_status);
+      break;
+    case LK_TC_COPY:
+      tc_copy_kernel<<<(unsigned)L.grid, 256, 0, s>>>((const CopyJob*)tab, (int)L.n_items, L.aux0,
+                                                     (uint16_t*)b.p[BASE_WORK], c->d_status);
       break;
     case LK_TC_GRAM:
     case LK_TC_PANEL: {

@@ -58,6 +58,10 @@ def tensor_block_map(tensors: Sequence[WL.Tensor]) -> List[List[int]]:
     return out
 
 
+CANARY = 7.25e9          # a value no optimizer quantity takes
+CANARY_WORDS = 256
+
+
 @dataclass
 class Tolerances:
     fp32: float = 1e-5       # elementwise / reduction paths
@@ -114,10 +118,36 @@ class ParityRun:
         self.host_params0 = host
         gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
         self.grads = torch.zeros(self.total, dtype=gdt, device=self.dev)
-        self.state = torch.zeros(self.ctx.adapm_state_bytes() // 4, dtype=torch.float32, device=self.dev)
-        self.work = torch.zeros(max(self.ctx.adapm_workspace_bytes() // 4, 64), dtype=torch.float32, device=self.dev)
+        # canary words: behind the state and the workspace, and in every gap between the state's sub-buffers
+        n_state = self.ctx.adapm_state_bytes() // 4
+        n_work = max(self.ctx.adapm_workspace_bytes() // 4, 64)
+        self._state_full = torch.zeros(n_state + CANARY_WORDS, dtype=torch.float32, device=self.dev)
+        self._work_full = torch.zeros(n_work + CANARY_WORDS, dtype=torch.float32, device=self.dev)
+        self.state, self.work = self._state_full[:n_state], self._work_full[:n_work]
         self.ctx.adapm_set_workspace(self.work)
         self.ctx.adapm_state_init(self.state)
+        self._state_full[n_state:] = CANARY
+        self._work_full[n_work:] = CANARY
+        used = []
+        for bi in range(len(self.blocks)):
+            for which in (A.STATE_M, A.STATE_L, A.STATE_R, A.STATE_V):
+                off, cnt = self.ctx.adapm_state_layout(bi, which)
+                if cnt > 0:
+                    used.append((off, off + cnt))
+        used.sort()
+        self._gaps, cur = [], 0
+        for a0, a1 in used:
+            assert a0 >= cur, "state sub-buffers overlap"
+            if a0 > cur:
+                self._gaps.append((cur, a0))
+            cur = a1
+        if cur < n_state:
+            self._gaps.append((cur, n_state))
+        if len(self._gaps) <= 4096:
+            for a0, a1 in self._gaps:
+                self.state[a0:a1] = CANARY
+        else:
+            self._gaps = []
         self.grad_scale = grad_scale
         self.shadow = None
         if shadow:
@@ -130,7 +160,8 @@ class ParityRun:
         oh = O.HParams(lr=f32(hpk["lr"]), beta1=f32(hpk["beta1"]), beta2=f32(hpk["beta2"]), eps=f32(hpk["eps"]),
                        clip=f32(hpk["clip"]), inner_iters=hpk["inner_iters"], inner_lr_scale=f32(hpk["inner_lr_scale"]),
                        adam_debias=bool(hpk.get("adam_debias", 0)), correction=bool(hpk.get("correction", 1)),
-                       max_grad_norm=(f32(hpk["max_grad_norm"]) if hpk.get("max_grad_norm", 0) > 0 else math.inf))
+                       max_grad_norm=(f32(hpk["max_grad_norm"]) if hpk.get("max_grad_norm", 0) > 0 else math.inf),
+                       refresh_period=max(1, int(hpk.get("refresh_period", 0))))
         self.ohp = oh
         self.ostate: Dict[int, O.BlockState] = {}
         self.oW: Dict[int, np.ndarray] = {}
@@ -258,8 +289,21 @@ class ParityRun:
                     assert em <= tol.fp32, f"block {bi} step {self.t}: m error {em:.3e}"
         return worst
 
+    def check_canaries(self) -> None:
+        """No kernel wrote behind the state or the workspace, or between two sub-buffers of the state."""
+        self.torch.cuda.synchronize()
+        n_state, n_work = self.state.numel(), self.work.numel()
+        assert bool((self._state_full[n_state:] == CANARY).all()), "a kernel wrote behind the state buffer"
+        assert bool((self._work_full[n_work:] == CANARY).all()), "a kernel wrote behind the workspace"
+        for a0, a1 in self._gaps:
+            assert bool((self._state_full[a0:a1] == CANARY).all()), f"a kernel wrote into the state gap [{a0}, {a1})"
+
     def close(self) -> None:
-        self.ctx.adapm_destroy()
+        try:
+            if getattr(self, "_state_full", None) is not None and self.state.data_ptr() == self._state_full.data_ptr():
+                self.check_canaries()
+        finally:
+            self.ctx.adapm_destroy()
 
 
 def sample_blocks(blocks: Sequence, per_class: int = 1) -> List[int]:

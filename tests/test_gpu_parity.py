@@ -553,3 +553,34 @@ def test_finite_check_skips_the_step_and_reports_it():
         assert run.ctx.adapm_get_status() == 0
     finally:
         run.close()
+
+
+# ------------------------------------------------------------------------------------ refresh period T
+
+@pytest.mark.parametrize("path", [A.PATH_TENSOR, A.PATH_SIMT])
+def test_refresh_period_holds_L_between_refreshes(path):
+    """refresh_period = 3: Algorithm 2 refits both factors at steps 1, 4, 7, ...; in between L stays as it is (bit
+    for bit) and only R is refitted.  Every step is compared with the oracle's reading of T."""
+    import torch
+    blocks = _pack([(300, 256, A.MOM_LOWRANK, 20, A.V_BLOCKMEAN, 1), (128, 640, A.MOM_LOWRANK, 6, A.V_ELEMENT, 0),
+                    (256, 512, A.MOM_LOWRANK, 16, A.V_BLOCKMEAN, 64), (64, 64, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1)])
+    w = WL.Workload("refresh", [], "bf16", "normal", steps=8)
+    run = ParityRun(w, True, lowrank_path=path, custom_blocks=blocks, hp_overrides=dict(refresh_period=3))
+    try:
+        for s in range(1, 9):
+            off, cnt = run.ctx.adapm_state_layout(0, A.STATE_L)
+            before = run.state[off:off + cnt].clone()
+            run.step()
+            run.compare()
+            torch.cuda.synchronize()
+            same = torch.equal(before, run.state[off:off + cnt])
+            assert same == ((s - 1) % 3 != 0), f"step {s}: L {'did not move' if same else 'moved'}"
+        assert run.ctx.adapm_get_status() == 0
+    finally:
+        run.close()
+
+
+def test_refresh_period_on_llama60m():
+    w = WL.get_workload("llama60m")
+    blocks, _ = A.adapm_plan_default(w.tensors)
+    _run(w, True, 9, sel=sample_blocks(blocks, 1), pooled=True, every=3, hp=dict(refresh_period=4))
