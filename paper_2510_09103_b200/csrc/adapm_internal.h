@@ -172,7 +172,8 @@ int launch_gemm(const GemmProb* d_tab, int64_t n_prob, int64_t n_tiles, const Ba
                 cudaStream_t s);
 int launch_apply_simt(const ApplyBlk* d_tab, int64_t n_blk, int64_t n_tiles, const Bases& b, const StepScalars& sc,
                       int grad_dtype, cudaStream_t s);
-int launch_copy_f32(float* dst, const float* src, int64_t n, const int32_t* status, cudaStream_t s);
+int launch_copy_ranges(const NormRange* d_tab, const int32_t* d_cta_range, int64_t n_ctas, float* dst, const float* src,
+                       const int32_t* status, cudaStream_t s);
 int launch_meansq_partial(const void* g, int grad_dtype, int64_t n_groups, int64_t group_elems, int chunks_per_group,
                           float* partial, cudaStream_t s);
 int launch_meansq_final(const float* partial, int64_t n_groups, int64_t group_elems, int chunks_per_group, float* out,

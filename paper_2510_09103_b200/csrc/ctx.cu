@@ -415,7 +415,22 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
       ab.push_back(a);
     }
     prog.push_back({LK_APPLY_SIMT, append_table(c->h_tables, ab), (int64_t)ab.size(), tiles});
-    if (c->final_lr_buf >= 0) prog.push_back({LK_COMMIT, 0, 0, 1});
+    if (c->final_lr_buf >= 0) {
+      // the refitted factors go back to the state, sub-buffer by sub-buffer (the padding between them is not touched)
+      std::vector<NormRange> ranges;
+      std::vector<int32_t> cta_range;
+      for (int64_t i : lowrank_ids) {
+        const adapm_block& b = c->blocks[i];
+        for (int which = 0; which < 2; ++which) {
+          NormRange r{which ? c->r_off[i] : c->l_off[i], (int64_t)b.rank * (which ? b.cols : b.rows), (int64_t)cta_range.size()};
+          for (int64_t q = 0; q < (r.numel + kNormChunk - 1) / kNormChunk; ++q) cta_range.push_back((int32_t)ranges.size());
+          ranges.push_back(r);
+        }
+      }
+      Launch CM{LK_COMMIT, append_table(c->h_tables, ranges), (int64_t)ranges.size(), (int64_t)cta_range.size()};
+      CM.aux0 = append_table(c->h_tables, cta_range);
+      prog.push_back(CM);
+    }
   }
   c->work_floats = work_cursor;
 
@@ -616,7 +631,9 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
       case LK_APPLY_SIMT:
         rc = launch_apply_simt((const ApplyBlk*)tab, L.n_items, L.grid, b, sc, hp.grad_dtype, s); break;
       case LK_COMMIT:
-        rc = launch_copy_f32((float*)state, work + c->ws_lr[c->final_lr_buf], c->lr_section_floats, c->d_status, s); break;
+        rc = launch_copy_ranges((const NormRange*)tab, (const int32_t*)(c->d_tables + L.aux0), L.grid, (float*)state,
+                                work + c->ws_lr[c->final_lr_buf], c->d_status, s);
+        break;
       default:
         rc = run_tensor_launch(c, L, b, sc, parity, s); break;
     }

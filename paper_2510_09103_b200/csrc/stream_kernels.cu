@@ -401,11 +401,23 @@ __global__ void __launch_bounds__(1024) gradnorm_final_kernel(const float* __res
   }
 }
 
-__global__ void copy_f32_kernel(float4* __restrict__ dst, const float4* __restrict__ src, int64_t n4,
-                                const int32_t* __restrict__ status) {
+// dst[off + i] = src[off + i] for the listed ranges only (one CTA per chunk of up to kNormChunk floats): the padding
+// between two sub-buffers of the state is never written
+__global__ void __launch_bounds__(256) copy_ranges_kernel(const NormRange* __restrict__ tab,
+                                                          const int32_t* __restrict__ cta_range, float* __restrict__ dst,
+                                                          const float* __restrict__ src,
+                                                          const int32_t* __restrict__ status) {
   if (*status != 0) return;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x)
-    dst[i] = src[i];
+  const NormRange R = tab[cta_range[blockIdx.x]];
+  const int64_t start = ((int64_t)blockIdx.x - R.first_cta) * kNormChunk;
+  const int64_t rem = R.numel - start;
+  const int len = rem < kNormChunk ? (int)rem : kNormChunk;
+  const float* s = src + R.off + start;
+  float* d = dst + R.off + start;
+  const int n4 = len / 4;                       // range offsets are multiples of 64 floats, chunks of 16384
+  for (int i = threadIdx.x; i < n4; i += 256)
+    reinterpret_cast<float4*>(d)[i] = reinterpret_cast<const float4*>(s)[i];
+  for (int i = 4 * n4 + threadIdx.x; i < len; i += 256) d[i] = s[i];
 }
 
 }  // namespace
@@ -498,13 +510,10 @@ int launch_gradnorm(const NormRange* d_tab, const int32_t* d_cta_range, int64_t 
   return ADAPM_OK;
 }
 
-int launch_copy_f32(float* dst, const float* src, int64_t n, const int32_t* status, cudaStream_t s) {
-  if (n <= 0) return ADAPM_OK;
-  // n is a multiple of 64 floats by construction of the state layout
-  const int64_t n4 = n / 4;
-  int64_t grid = (n4 + 255) / 256;
-  if (grid > 148 * 16) grid = 148 * 16;
-  copy_f32_kernel<<<(unsigned)grid, 256, 0, s>>>((float4*)dst, (const float4*)src, n4, status);
+int launch_copy_ranges(const NormRange* d_tab, const int32_t* d_cta_range, int64_t n_ctas, float* dst, const float* src,
+                       const int32_t* status, cudaStream_t s) {
+  if (n_ctas <= 0) return ADAPM_OK;
+  copy_ranges_kernel<<<(unsigned)n_ctas, 256, 0, s>>>(d_tab, d_cta_range, dst, src, status);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }
