@@ -76,10 +76,6 @@ def recorded_traffic(kind: str, workload: str, v_mode: str):
 
 # ------------------------------------------------------------------------------------------------ oracle arm
 
-def _class_key(b):
-    return (b.mom_mode, b.rows, b.cols, b.rank, b.v_mode, b.v_group_rows)
-
-
 def _oracle_hparams(w):
     from oracle import adapm_oracle as O
     return O.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
@@ -169,45 +165,6 @@ def oracle_layer_sample(w, blocks, budget_s: float = 25.0):
             f"({sample.elems} of {sum(b.rows * b.cols for b in blocks)} elements), one oracle step; layer time x "
             f"{n_layers}, embeddings by element count")
     return est_all, est_one, desc
-
-
-def oracle_step_estimate(w, blocks, max_rows: int = 4096, seed: int = 0):
-    """Time one oracle step on one block of every class and scale by the class sizes.
-
-    Returns (estimated seconds for a full step, description of the sample).  Blocks with more than
-    `max_rows` rows and no low-rank factors are timed on their first `max_rows` rows and scaled.
-    """
-    from oracle import adapm_oracle as O
-    import workloads as WL
-    classes = {}
-    for i, b in enumerate(blocks):
-        classes.setdefault(_class_key(b), []).append(i)
-    hp = O.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps)
-    rng = np.random.default_rng(seed)
-    total, sampled_elems = 0.0, 0
-    for key, ids in classes.items():
-        b = blocks[ids[0]]
-        rows = b.rows
-        scale = 1.0
-        if b.mom_mode != O.MOM_LOWRANK and rows > max_rows:
-            gr = max(b.v_group_rows, 1)
-            rows = max_rows // gr * gr
-            scale = b.rows / rows
-        ob = O.Block(rows, b.cols, b.mom_mode, b.rank, b.v_mode, b.v_group_rows, b.lr_scale, b.weight_decay)
-        L0 = O.init_L0(rows, b.rank, 0, ids[0]) if b.mom_mode == O.MOM_LOWRANK else None
-        st = O.new_state(ob, L0)
-        W = rng.standard_normal((rows, b.cols)) * 0.02
-        g, _ = WL.to_grad_dtype((rng.standard_normal((rows, b.cols)) * 1e-3).astype(np.float32), w.grad_dtype)
-        g = g.astype(np.float64)
-        t0 = time.perf_counter()
-        O.block_step(W, g, st, ob, hp, 1)
-        dt = time.perf_counter() - t0
-        total += dt * scale * len(ids)
-        sampled_elems += rows * b.cols
-    desc = (f"one block of each of {len(classes)} block classes (non-low-rank blocks capped at {max_rows} rows), "
-            f"{sampled_elems} of {sum(b.rows * b.cols for b in blocks)} elements, one step each, "
-            f"scaled by class size")
-    return total, desc
 
 
 def _blas_threads() -> int:
