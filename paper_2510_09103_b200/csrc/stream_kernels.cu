@@ -86,36 +86,13 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
     }
   }
 
-  float v_group = 0.f;
-  if (B.v_mode == SV_GROUP_INLINE) {
-    // one thread reads the old scalar and writes the new one; everyone else gets it by broadcast
-    float v_old = 0.f;
-    if (lane == 0) v_old = state[B.v_off + group];
-    const float tot = team_sum<TEAM>(ss, smem8);
-    if (TEAM == 32) {
-      v_old = __shfl_sync(0xffffffffu, v_old, 0);
-    } else {
-      if (threadIdx.x == 0) smem8[8] = v_old;
-      __syncthreads();
-      v_old = smem8[8];
-    }
-    v_group = sc.beta2 * v_old + (1.f - sc.beta2) * ((gs * gs) * (tot / (float)ulen));
-    if (lane == 0) state[B.v_off + group] = v_group;
-  } else if (B.v_mode == SV_GROUP_READY) {
-    v_group = state[B.v_off + group];
-  }
-
   // ---- phase 2: momentum, second moment, parameter write ------------------------------------
   // Chunks are taken four at a time: all loads of a batch are issued before its first store, so the
-  // memory system sees them together instead of one round trip per chunk.
-  const float lr_s = sc.lr * B.lr_scale;
-  const float a1 = 1.f - sc.beta1, a2 = 1.f - sc.beta2;
-  // with a group scalar the division m^c / (sqrt(v) + eps) is one multiplication per element
-  const float k_ratio = sc.inv_bc1 / (sqrtf(v_group * sc.inv_bc2) + sc.eps);
+  // memory system sees them together instead of one round trip per chunk.  The first batch is asked
+  // for before the group mean is reduced: its W (and m, v) do not depend on the mean, and the round
+  // trip of the reduction's shuffles and of the old group scalar then overlaps theirs.
   constexpr int kBatch = ((HAS_M && HAS_V) || sizeof(typename GT::raw8) > 16) ? 2 : 4;
-#pragma unroll
-  for (int c0 = 0; c0 < kTeamChunks; c0 += kBatch) {
-    float w[kBatch][8], m[kBatch][8], v[kBatch][8];
+  auto load_batch = [&](int c0, float (*w)[8], float (*m)[8], float (*v)[8]) {
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       const int idx = lane + (c0 + b) * TEAM;
@@ -136,6 +113,47 @@ __device__ __forceinline__ void run_unit(const StreamBlk& B, int64_t unit, float
           }
         }
       }
+    }
+  };
+  float w[kBatch][8], m[kBatch][8], v[kBatch][8];
+  load_batch(0, w, m, v);
+
+  float v_group = 0.f;
+  if (B.v_mode == SV_GROUP_INLINE) {
+    // one thread reads the old scalar and writes the new one; everyone else gets it by broadcast
+    float v_old = 0.f;
+    if (lane == 0) v_old = state[B.v_off + group];
+    const float tot = team_sum<TEAM>(ss, smem8);
+    if (TEAM == 32) {
+      v_old = __shfl_sync(0xffffffffu, v_old, 0);
+    } else {
+      if (threadIdx.x == 0) smem8[8] = v_old;
+      __syncthreads();
+      v_old = smem8[8];
+    }
+    v_group = sc.beta2 * v_old + (1.f - sc.beta2) * ((gs * gs) * (tot / (float)ulen));
+    if (lane == 0) state[B.v_off + group] = v_group;
+  } else if (B.v_mode == SV_GROUP_READY) {
+    v_group = state[B.v_off + group];
+  }
+
+  const float lr_s = sc.lr * B.lr_scale;
+  const float a1 = 1.f - sc.beta1, a2 = 1.f - sc.beta2;
+  // with a group scalar the division m^c / (sqrt(v) + eps) is one multiplication per element
+  const float k_ratio = sc.inv_bc1 / (sqrtf(v_group * sc.inv_bc2) + sc.eps);
+  // Blocks without momentum and with a group scalar hold only W per chunk: their second batch is requested
+  // before the first is worked on (two register sets that swap roles).
+  constexpr bool kTwoSets = !HAS_M && !HAS_V && kBatch * 2 == kTeamChunks;
+  float w2[kTwoSets ? kBatch : 1][8];
+  if (kTwoSets) load_batch(kBatch, w2, m, v);
+#pragma unroll
+  for (int c0 = 0; c0 < kTeamChunks; c0 += kBatch) {
+    if (c0 > 0 && !kTwoSets) load_batch(c0, w, m, v);
+    if (c0 > 0 && kTwoSets) {
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[b][i] = w2[b][i];
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
