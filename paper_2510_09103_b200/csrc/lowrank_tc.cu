@@ -444,7 +444,18 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
   // ---- refit passes, once per parity of the step and per kind of step ------------------------------------------
   // With a refresh period T > 1 a step either refits both factors (phase 1) or holds L and refits R (phase 2:
   // Gram matrices of L only, column panels only, and the split copy of L carried over to the final set).
-  const int team_mode = (hp.flags & ADAPM_FLAG_NO_PANEL_TEAMS) ? 1 : ((hp.flags & ADAPM_FLAG_FORCE_PANEL_TEAMS) ? 2 : 0);
+  int team_mode = (hp.flags & ADAPM_FLAG_NO_PANEL_TEAMS) ? 1 : ((hp.flags & ADAPM_FLAG_FORCE_PANEL_TEAMS) ? 2 : 0);
+  {
+    // The team pacing lets CTAs of a launch wait for one another, which is only sound when the whole grid (at most
+    // one CTA per SM) can be resident at once: ask the runtime whether an SM takes a CTA of this size at all (a
+    // device or an MPS share with less shared memory or fewer registers does not), else hand items out longest-first.
+    int resident = 0;
+    cudaFuncSetAttribute(tc::tc_items_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P->smem_engine);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, tc::tc_items_kernel, tc::kEngineThreads,
+                                                      (size_t)P->smem_engine) != cudaSuccess || resident < 1)
+      team_mode = 1;
+    (void)cudaGetLastError();
+  }
   const bool with_hold = hp.refresh_period > 1 && K_eff > 0;
   for (int parity = 0; parity < (P->rotate ? 2 : 1); ++parity)
   for (int phase = (with_hold ? 1 : 0); phase <= (with_hold ? 2 : 0); ++phase) {

@@ -26,11 +26,11 @@
 //      loads, not the tensor pipe, bound this kernel)
 //   B  one 3-D box: stage_k rows x (64 x chunks) columns of a [rows, 2 half] array, i.e. the N side
 //      read MN-major with its 64-column chunks one box apart
-// Warp roles (384 threads): warp 0 issues the TMA loads of a stage, warp 1 issues its MMAs, warps
-// 2 and 3 add up g^2 per row from the gradient tiles of the first segment when the launch asks for
-// it (the second-moment statistic of the block-mean form then needs no pass of its own over g),
-// warps 4-11 drain the accumulators (two groups of four warps that take the 16-column pieces of an
-// item alternately).  The two issuing threads run dependent scalar code, so their per-stage instruction
+// Warp roles (512 threads, 128 registers each): warp 0 issues the TMA loads of a stage, warp 1 issues
+// its MMAs, warps 4-7 add up g^2 per row from the gradient tiles of the first segment when the
+// launch asks for it (the second-moment statistic of the block-mean form then needs no pass of its
+// own over g), warps 8-15 drain the accumulators (two groups of four warps that take the 16-column
+// pieces of an item alternately); warps 2 and 3 have no work.  The two issuing threads run dependent scalar code, so their per-stage instruction
 // count is what bounds the rate; both loops are kept short.  With two accumulator buffers the
 // epilogue of one item overlaps the K-loops of the next.  Every wait is bounded; when one runs out
 // the CTA records a status bit, stops taking work and leaves through the common exit (which frees
@@ -46,7 +46,7 @@ namespace tc {
 
 constexpr int kMaxSegs = 4;
 constexpr int kMaxA = 3;
-constexpr int kEngineThreads = 384;
+constexpr int kEngineThreads = 512;
 constexpr uint32_t kTeamSpinDefault = 1u << 22;   // polls of 256 ns each: about a second
 constexpr uint32_t kWaitSpinDefault = 1u << 23;   // mbarrier polls: at least as long as a team wait
 
@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
   const uint32_t wlim = a.wait_spin_limit;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 8; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], a.sumsq_on ? 3 : 1); }
+    for (int i = 0; i < 8; ++i) { mbar_init(&sh.full[i], 1); mbar_init(&sh.empty[i], a.sumsq_on ? 5 : 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.tfull[i], 1); mbar_init(&sh.tempty[i], 256); }
     sh.abort = 0;
     mbar_fence_init();
@@ -334,10 +334,12 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       }
     }
   } else if (warp < 4) {
+    // no work
+  } else if (warp < 8) {
     // ------------------------------------------------------------------ row sums of g^2
-    // The two warps follow every stage of the launch (their arrivals are part of each stage's release); for an
-    // item with sumsq_off >= 0 they read the gradient tiles of the first segment (K along x), warp 2 the upper
-    // 64 rows of every panel, warp 3 the lower.  Eight lanes share a row of a box (its eight 16-byte pieces,
+    // The four warps follow every stage of the launch (their arrivals are part of each stage's release); for an
+    // item with sumsq_off >= 0 they read the gradient tiles of the first segment (K along x), each warp 32 rows
+    // of every panel.  Eight lanes share a row of a box (its eight 16-byte pieces,
     // whatever order the swizzle put them in), so a warp reads four rows per access without bank conflicts; a
     // lane keeps one partial sum per row it visits, and the eight partial sums of a row are added in a fixed
     // order at the end of the item.
@@ -345,15 +347,15 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      const int rsub = 64 * (warp - 2) + (lane >> 3), piece = lane & 7;
+      const int rsub = 32 * (warp - 4) + (lane >> 3), piece = lane & 7;
       for (int it = it_begin; it < it_end && ok; ++it) {
         const Item& I = a.items[it];
         const bool mine = I.sumsq_off >= 0;
-        float acc[kMaxA][16];
+        float acc[kMaxA][8];
 #pragma unroll
         for (int p = 0; p < kMaxA; ++p)
 #pragma unroll
-          for (int i = 0; i < 16; ++i) acc[p][i] = 0.f;
+          for (int i = 0; i < 8; ++i) acc[p][i] = 0.f;
         int n_a0 = 0;
         for (int s = 0; s < I.n_seg && ok; ++s) {
           const int k = I.seg[s].k, n_a = I.seg[s].n_a;
@@ -373,7 +375,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
                   for (int jb = 0; jb < n_box; ++jb) {
                     const uint8_t* box = sa + p * a_tile + jb * kBoxBytes + piece * 16;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
+                    for (int i = 0; i < 8; ++i) {
                       const uint4 v = *reinterpret_cast<const uint4*>(box + (4 * i + rsub) * 128);
                       const uint32_t w[4] = {v.x, v.y, v.z, v.w};
                       float s2 = acc[p][i];
@@ -400,7 +402,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
           for (int p = 0; p < kMaxA; ++p) {
             if (p < n_a0) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
+              for (int i = 0; i < 8; ++i) {
                 float s2 = acc[p][i];
                 s2 += __shfl_xor_sync(0xffffffffu, s2, 1);
                 s2 += __shfl_xor_sync(0xffffffffu, s2, 2);
@@ -417,7 +419,7 @@ __global__ void __launch_bounds__(kEngineThreads, 1) tc_items_kernel(EngineArgs 
     // ------------------------------------------------------------------ epilogue
     const int q = 32 * (warp & 3) + lane;               // accumulator row (= TMEM lane) of this thread
     const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
-    const int grp = (warp - 4) >> 2;                    // the two groups take the pieces of an item alternately
+    const int grp = (warp - 8) >> 2;                    // the two groups take the pieces of an item alternately
     const float gs = a.gscale ? *a.gscale : 1.f;
     int j = 0;
     for (int it = it_begin; it < it_end; ++it, ++j) {
