@@ -47,7 +47,8 @@ enum {
   MAP_GS = 20,      // + which: Gram operands as chunks
   MAP_W = 24, MAP_G32 = 25, MAP_V = 26,          // W, g, v in quarter-tile boxes (apply)
   MAP_LCAT = 27, MAP_RCAT = 28,                  // X and Y side by side as one matrix (apply)
-  kMapsPerBlock = 29
+  MAP_SH = 29,                                   // the bf16 copy of W, boxes like g's (apply; zero without a shadow)
+  kMapsPerBlock = 30
 };
 
 struct ConvertJob {
@@ -132,7 +133,7 @@ struct TcBlock {
 };
 
 struct MapSet {                     // tensor maps for one combination of caller buffers
-  const void* key[4] = {nullptr, nullptr, nullptr, nullptr};
+  const void* key[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // params, grads, state, workspace, shadow
   CUtensorMap* d_maps = nullptr;
   std::vector<CUtensorMap> h_maps;
   uint64_t last_use = 0;
@@ -606,7 +607,7 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           a.off = b.offset; a.v_off = c->v_off[t.id]; a.rows = b.rows; a.cols = b.cols; a.r = b.rank; a.rp = t.rp;
           a.half = t.half;
           a.map_l = mb + MAP_LCAT; a.map_r = mb + MAP_RCAT;
-          a.map_w = mb + MAP_W; a.map_g = mb + MAP_G32; a.map_v = mb + MAP_V;
+          a.map_w = mb + MAP_W; a.map_g = mb + MAP_G32; a.map_v = mb + MAP_V; a.map_sh = mb + MAP_SH;
           a.row0 = p0;
           a.tile0 = (int)((int64_t)tiles * q / runs);
           a.n_tiles = (int)((int64_t)tiles * (q + 1) / runs) - a.tile0;
@@ -697,7 +698,9 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, int64_t t, cudaStream_t s,
   ++P->use_clock;
   MapSet* slot = nullptr;
   for (MapSet& m : P->maps)
-    if (m.key[0] == b.p[0] && m.key[1] == b.p[1] && m.key[2] == b.p[2] && m.key[3] == b.p[3] && m.key[0]) slot = &m;
+    if (m.key[0] == b.p[0] && m.key[1] == b.p[1] && m.key[2] == b.p[2] && m.key[3] == b.p[3] && m.key[4] == b.shadow &&
+        m.key[0])
+      slot = &m;
   if (slot) {
     slot->last_use = P->use_clock;
     P->cur_maps = slot->d_maps;
@@ -736,6 +739,10 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, int64_t t, cudaStream_t s,
     }
     ok = ok && tc::encode_bf16_matrix(&m[MAP_LCAT], work + t2.lc[0] * 2, rows, 4 * half, 4 * half, 128);
     ok = ok && tc::encode_bf16_matrix(&m[MAP_RCAT], work + t2.rtc[0] * 2, cols, 4 * half, 4 * half, 128);
+    if (b.shadow)
+      ok = ok && tc::encode_panel32(&m[MAP_SH], reinterpret_cast<const char*>(b.shadow) + blk.offset * 2, rows, cols, false);
+    else
+      std::memset(&m[MAP_SH], 0, sizeof(CUtensorMap));
     for (int q = 0; q < 4; ++q)
       ok = ok && tc::encode_bf16_chunked(&m[MAP_GS + q], work + t2.gs[q] * 2, 2 * half, 2 * half, nb, sk);
     if (!ok) {
@@ -746,6 +753,7 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, int64_t t, cudaStream_t s,
   ADAPM_CUDA(cudaMemcpyAsync(slot->d_maps, slot->h_maps.data(), slot->h_maps.size() * sizeof(CUtensorMap),
                              cudaMemcpyHostToDevice, s));
   for (int q = 0; q < 4; ++q) slot->key[q] = b.p[q];
+  slot->key[4] = b.shadow;
   slot->last_use = P->use_clock;
   P->cur_maps = slot->d_maps;
   return ADAPM_OK;
@@ -799,7 +807,7 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       a.parity = parity;
       a.buf_bytes = P->apply_buf_bytes;
       a.gscale = b.gscale;
-      a.shadow = b.shadow;
+      a.shadow = b.shadow != nullptr;
       if (L.aux0 == 0) {
         a.r_region_off = P->apply_r_region; a.n_rstages = P->apply_r_stages;
         a.w_region_off = P->apply_w_region; a.n_bufs = P->apply_bufs;

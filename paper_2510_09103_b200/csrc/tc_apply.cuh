@@ -54,6 +54,7 @@ struct ApplyItem {
                              // = [hi0 | lo0 | hi1 | lo1], boxes of 64 x 128
   int32_t map_w, map_g;      // params and grads of the block, boxes of 32 x 128
   int32_t map_v;             // per-element v of the block (same boxes as params); unused with a group v
+  int32_t map_sh;            // bf16 copy of the params (same boxes as grads); used when the launch has a shadow
   int32_t row0;              // first row of the panel
   int32_t tile0, n_tiles;    // column tiles [tile0, tile0 + n_tiles) of 128 columns
   int32_t nbc1, nbc2;        // 64-wide boxes across the 2rp columns of the previous set / the 4rp of both
@@ -71,7 +72,7 @@ struct ApplyArgs {
   int32_t use_new;           // 0: c1 == 0, the refitted factors are not needed
   int32_t parity;            // 0: the left half of the operands holds the previous factors, 1: the right half
   const float* gscale;       // device scalar: every gradient counts as gscale[0] * g (nullptr: 1)
-  uint16_t* shadow;          // bf16 copy of the parameters, written with W (nullptr: none)
+  int32_t shadow;            // 1: the bf16 copy of the parameters is written with W (ApplyItem::map_sh)
   int32_t r_region_off;      // byte offset of the R ring inside the dynamic shared memory
   int32_t n_rstages;         // R ring depth (1..kApplyMaxStages); a stage is one 64 x 128 box of R^T
   int32_t w_region_off;      // byte offset of the g / W ring
@@ -306,6 +307,7 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           if (col < I.cols) {
             const uint8_t* buf = smem_w + (size_t)b * a.buf_bytes;
             tma_store_box(a.maps + I.map_w, col, I.row0, buf);
+            if (a.shadow) tma_store_box(a.maps + I.map_sh, col, I.row0, buf + kWBoxBytes);
             if (I.v_mode == ADAPM_V_ELEMENT) tma_store_box(a.maps + I.map_v, col, I.row0, buf + kApplyBufBytes);
           }
           bulk_commit_group();
@@ -418,13 +420,11 @@ __global__ void __launch_bounds__(kApplyThreads, 1) tc_apply_kernel(ApplyArgs a)
           shw[2 * i + 1] = pack_bf16x2(w[2], w[3]);
         }
         if (a.shadow) {
-          // this thread's 16 columns of the row as bf16: two 16-byte stores (columns come in groups of 8)
-          const int col = (I.tile0 + (q >> 2)) * kApplyNT + sub * kApplyQC + 16 * half;
-          if (rok) {
-            uint16_t* sp = a.shadow + I.off + (int64_t)row * I.cols + col;
-            if (col < I.cols) *reinterpret_cast<uint4*>(sp) = make_uint4(shw[0], shw[1], shw[2], shw[3]);
-            if (col + 8 < I.cols) *reinterpret_cast<uint4*>(sp + 8) = make_uint4(shw[4], shw[5], shw[6], shw[7]);
-          }
+          // The bf16 copy of the new W takes the place of the gradient in the buffer (this thread's two 16-byte
+          // pieces, already read): it has g's box shape and swizzle, and the mover stores it with the same kind of
+          // tensor map.
+          *reinterpret_cast<uint4*>(buf + g_at[0]) = make_uint4(shw[0], shw[1], shw[2], shw[3]);
+          *reinterpret_cast<uint4*>(buf + g_at[1]) = make_uint4(shw[4], shw[5], shw[6], shw[7]);
         }
         // one arrival per warp: every lane orders its own writes (and tensor-memory reads), the warp meets
         fence_async_smem();

@@ -30,8 +30,8 @@
 // its MMAs, warps 4-7 add up g^2 per row from the gradient tiles of the first segment when the
 // launch asks for it (the second-moment statistic of the block-mean form then needs no pass of its
 // own over g), warps 8-15 drain the accumulators (two groups of four warps that take the 16-column
-// pieces of an item alternately); warps 2 and 3 have no work.  The two issuing threads run dependent scalar code, so their per-stage instruction
-// count is what bounds the rate; both loops are kept short.  With two accumulator buffers the
+// pieces of an item alternately); warps 2 and 3 have no work.  The two issuing threads run dependent
+// scalar code, so their per-stage instruction count is what bounds the rate; both loops are kept short.  With two accumulator buffers the
 // epilogue of one item overlaps the K-loops of the next.  Every wait is bounded; when one runs out
 // the CTA records a status bit, stops taking work and leaves through the common exit (which frees
 // its tensor memory).  A launch that finds the status word set on entry does nothing.
@@ -119,7 +119,7 @@ struct EngineArgs {
   int32_t n_acc;             // 1 or 2 accumulator buffers
   const int32_t* cta_begin;  // CTA c runs items [cta_begin[c], cta_begin[c + 1]) in order
   int32_t sum_col;           // EPI_FACTOR: first of the tensor-memory columns the epilogue parks D0 + D1 in, or -1
-  int32_t sumsq_on;          // 1: warp 10 follows the stages and sums g^2 for items that have sumsq_off >= 0
+  int32_t sumsq_on;          // 1: warps 4-7 follow the stages and sum g^2 for items that have sumsq_off >= 0
   int32_t* team_counters;    // one counter per team, zero at launch (nullptr when no item waits)
   uint32_t team_spin_limit, wait_spin_limit;
   const float* gscale;       // device scalar: every gradient counts as gscale[0] * g (nullptr: 1)
