@@ -73,6 +73,27 @@ def test_create_rejects_bad_descriptors_on_the_host():
     assert _create_code([ok], beta1=1.0) == -3
     assert _create_code([ok], grad_dtype=9) == -1
     assert _create_code([ok], inner_iters=-1) == -3
+    assert _create_code([ok], refresh_period=-1) == -3
+    assert _create_code([ok], max_grad_norm=-1.0) == -3
+    assert _create_code([ok], max_grad_norm=float("nan")) == -3
+    assert _create_code([ok], tune_stage_k=32) == -3
+    assert _create_code([ok], tune_panels=4) == -3
+
+
+def test_hparams_struct_matches_the_header():
+    """The ctypes mirror of adapm_hparams lists the header's fields in the header's order."""
+    text = open(os.path.join(ROOT, "include", "adapm.h")).read()
+    body = text[text.index("typedef struct {\n  float   lr, beta1"):text.index("} adapm_hparams;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    names = []
+    for decl in body.split(";"):
+        decl = decl.replace("typedef struct {", "").strip()
+        if not decl:
+            continue
+        first, *rest = decl.split(",")
+        names.append(first.split()[-1])
+        names += [r.strip() for r in rest]
+    assert names == [f for f, _ in A.adapm_hparams._fields_]
 
 
 def test_planner_rejects_bad_input():

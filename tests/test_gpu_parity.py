@@ -476,12 +476,16 @@ def test_llama3_8b_block_shapes_on_the_tensor_path():
 
 @pytest.mark.parametrize("pct", [2, 10, 50])
 def test_rank_ratios_of_the_ablation(pct):
-    """Section 5.1.2 sweeps the rank over 2, 5, 10 and 50 percent of the full rank; at d = 1024 that is 20, 102 and
-    512.  Up to rank 256 the blocks run on the tensor path, above on the CUDA-core path (AUTO)."""
+    """Section 5.1.2 sweeps the rank over 2, 5, 10 and 50 percent of the full rank; on the LLaMA-350M block shapes
+    (d = 1024, FFN 2736) that is 20, 102 and 512.  Up to rank 256 the blocks run on the tensor path, above on the
+    CUDA-core path (AUTO).  The ranks come from the planner; the blocks are one of each low-rank shape."""
     w = WL.get_workload("llama350m", rank_pct=pct)
-    blocks, _ = A.adapm_plan_default(w.tensors, rank_pct=pct)
-    sel = [i for i in sample_blocks(blocks, 1) if blocks[i].mom_mode == A.MOM_LOWRANK and blocks[i].rows <= 1024]
-    _run(w, True, 4, sel=sel, pooled=True, every=2)
+    planned, _ = A.adapm_plan_default(w.tensors, rank_pct=pct)
+    shapes = sorted({(b.rows, b.cols, b.rank, b.v_group_rows) for b in planned if b.mom_mode == A.MOM_LOWRANK})
+    want = max(1, pct * 1024 // 100)
+    assert shapes == [(1024, 1024, want, 64), (1024, 2736, want, 1), (2736, 1024, want, 1)]
+    blocks = _pack([(r, c, A.MOM_LOWRANK, k, A.V_BLOCKMEAN, g) for r, c, k, g in shapes])
+    _run(WL.Workload(f"ratio{pct}", [], "bf16", "heavyrows", steps=4), True, 4, blocks=blocks)
 
 
 # ------------------------------------------------------------------------------------ global clipping, bf16 copy, finite check
