@@ -702,7 +702,12 @@ extern "C" int adapm_get_status(adapm_ctx* c, adapm_stream stream, int32_t* stat
   int32_t h = 0;
   ADAPM_CUDA(cudaMemcpyAsync(&h, c->d_status, sizeof(h), cudaMemcpyDeviceToHost, s));
   ADAPM_CUDA(cudaStreamSynchronize(s));
-  if (h != 0) ADAPM_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(h), s));
+  if (h != 0) {
+    ADAPM_CUDA(cudaMemsetAsync(c->d_status, 0, sizeof(h), s));
+    // steps issued while the word was set wrote nothing, so the bf16 copies of the factors no longer follow the
+    // step numbers the host has counted: rebuild them from the state at the next step
+    tensor_state_changed(c);
+  }
   *status = h;
   return h == 0 ? ADAPM_OK : ADAPM_EDEVICE;
 }

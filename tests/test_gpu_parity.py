@@ -554,6 +554,16 @@ def test_finite_check_skips_the_step_and_reports_it():
         assert run.ctx.adapm_get_status() == A.ST_NONFINITE_GRAD
         run.step()
         run.compare()
+        # a caller that counts the skipped step and goes on with the next number must get the same result as one
+        # that repeats the number: the library rebuilds its bf16 copies of the factors after a reported skip
+        before = run.params.clone(), run.state.clone()
+        run.ctx.adapm_step(run.params, bad, run.state, run.t + 1)
+        torch.cuda.synchronize()
+        assert torch.equal(before[0], run.params) and torch.equal(before[1], run.state)
+        assert run.ctx.adapm_get_status() == A.ST_NONFINITE_GRAD
+        run.t += 1                      # the skipped step keeps its number
+        run.step()
+        run.compare()
         assert run.ctx.adapm_get_status() == 0
     finally:
         run.close()
