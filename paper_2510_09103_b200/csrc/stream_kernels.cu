@@ -304,25 +304,53 @@ __device__ __forceinline__ float warp_sum_partials(const float* __restrict__ p, 
   return s;
 }
 
+// One warp per group, or (kLane) one lane per group for jobs whose groups have few partial sums: a lane then
+// adds its group's partial sums one after the other.  Either way the order of the additions is fixed.
+constexpr int kLaneGroupMax = 64;     // partial sums per group up to which a lane takes a whole group
+
 __global__ void __launch_bounds__(256) reduce_final_kernel(const ReduceJob* __restrict__ tab, int n_jobs,
                                                            int64_t n_groups, float* __restrict__ state,
                                                            const float* __restrict__ work, float beta2,
                                                            const int32_t* __restrict__ status,
                                                            const float* __restrict__ gscale) {
-  const int64_t gidx = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (gidx >= n_groups || *status != 0) return;
+  // groups are taken 32 at a time by a warp; inside the 32, jobs with small groups go lane by lane
+  const int64_t g0 = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * 32;
+  if (g0 >= n_groups || *status != 0) return;
+  const int lane = threadIdx.x & 31;
+  const float gs2 = gscale ? gscale[1] : 1.f;      // the sums are of the unclipped gradient
   int lo = 0, hi = n_jobs - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
-    if (tab[mid].first_group <= gidx) lo = mid; else hi = mid - 1;
+    if (tab[mid].first_group <= g0) lo = mid; else hi = mid - 1;
   }
-  const ReduceJob J = tab[lo];
-  const int64_t group = gidx - J.first_group;
-  const float tot = warp_sum_partials(work + J.part_off + group * J.chunks_per_group, J.chunks_per_group);
-  if ((threadIdx.x & 31) == 0) {
-    float* v = state + J.v_off + group;
-    const float gs2 = gscale ? gscale[1] : 1.f;      // the sums are of the unclipped gradient
-    *v = beta2 * (*v) + (1.f - beta2) * (gs2 * (tot / (float)J.group_elems));
+  const int64_t g_end = g0 + 32 < n_groups ? g0 + 32 : n_groups;
+  int64_t g = g0;
+  while (g < g_end) {                                // warp-uniform walk over the jobs these 32 groups fall in
+    while (lo + 1 < n_jobs && tab[lo + 1].first_group <= g) ++lo;
+    const ReduceJob J = tab[lo];
+    const int64_t job_end = J.first_group + J.n_groups;
+    const int64_t upto = job_end < g_end ? job_end : g_end;
+    if (J.chunks_per_group <= kLaneGroupMax) {
+      const int64_t mine = g + lane;
+      if (mine < upto) {
+        const int64_t group = mine - J.first_group;
+        const float* p = work + J.part_off + group * J.chunks_per_group;
+        float tot = 0.f;
+        for (int i = 0; i < J.chunks_per_group; ++i) tot += p[i];
+        float* v = state + J.v_off + group;
+        *v = beta2 * (*v) + (1.f - beta2) * (gs2 * (tot / (float)J.group_elems));
+      }
+    } else {
+      for (int64_t q = g; q < upto; ++q) {
+        const int64_t group = q - J.first_group;
+        const float tot = warp_sum_partials(work + J.part_off + group * J.chunks_per_group, J.chunks_per_group);
+        if (lane == 0) {
+          float* v = state + J.v_off + group;
+          *v = beta2 * (*v) + (1.f - beta2) * (gs2 * (tot / (float)J.group_elems));
+        }
+      }
+    }
+    g = upto;
   }
 }
 
@@ -483,8 +511,8 @@ int launch_reduce_partial(const ReduceJob* d_tab, const int32_t* d_cta_job, int6
 int launch_reduce_final(const ReduceJob* d_tab, int64_t n_jobs, int64_t n_groups, float* state, const float* work,
                         float beta2, const int32_t* status, const float* gscale, cudaStream_t s) {
   if (n_groups <= 0) return ADAPM_OK;
-  reduce_final_kernel<<<(unsigned)((n_groups + 7) / 8), 256, 0, s>>>(d_tab, (int)n_jobs, n_groups, state, work, beta2,
-                                                                    status, gscale);
+  reduce_final_kernel<<<(unsigned)((n_groups + 255) / 256), 256, 0, s>>>(d_tab, (int)n_jobs, n_groups, state, work, beta2,
+                                                                        status, gscale);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }
