@@ -22,8 +22,7 @@
 // A stage of the shared-memory ring holds `stage_k` (64 or 128) of K:
 //   A  up to three operands of 128 rows x stage_k (K along x: boxes of 64 x 128) or stage_k x 128
 //      columns (K along y: two boxes of 64 x stage_k).  All are multiplied with the same B and fill
-//      one accumulator each: the more operands share a B, the fewer bytes a flop brings in (the
-//      loads, not the tensor pipe, bound this kernel)
+//      one accumulator each: the more operands share a B, the fewer bytes a flop brings in
 //   B  one 3-D box: stage_k rows x (64 x chunks) columns of a [rows, 2 half] array, i.e. the N side
 //      read MN-major with its 64-column chunks one box apart
 // Warp roles (512 threads, 128 registers each): warp 0 issues the TMA loads of a stage, warp 1 issues
@@ -31,8 +30,8 @@
 // launch asks for it (the second-moment statistic of the block-mean form then needs no pass of its
 // own over g), warps 8-15 drain the accumulators (two groups of four warps that take the 16-column
 // pieces of an item alternately); warps 2 and 3 have no work.  The two issuing threads run dependent
-// scalar code, so their per-stage instruction count is what bounds the rate; both loops are kept short.  With two accumulator buffers the
-// epilogue of one item overlaps the K-loops of the next.  Every wait is bounded; when one runs out
+// scalar code, so their per-stage instruction count is what bounds the rate; both loops are kept
+// short.  With two accumulator buffers the epilogue of one item overlaps the K-loops of the next.  Every wait is bounded; when one runs out
 // the CTA records a status bit, stops taking work and leaves through the common exit (which frees
 // its tensor memory).  A launch that finds the status word set on entry does nothing.
 #pragma once
