@@ -31,9 +31,10 @@
 // own over g), warps 8-15 drain the accumulators (two groups of four warps that take the 16-column
 // pieces of an item alternately); warps 2 and 3 have no work.  The two issuing threads run dependent
 // scalar code, so their per-stage instruction count is what bounds the rate; both loops are kept
-// short.  With two accumulator buffers the epilogue of one item overlaps the K-loops of the next.  Every wait is bounded; when one runs out
-// the CTA records a status bit, stops taking work and leaves through the common exit (which frees
-// its tensor memory).  A launch that finds the status word set on entry does nothing.
+// short.  With two accumulator buffers the epilogue of one item overlaps the K-loops of the next.
+// Every wait is bounded; when one runs out the CTA records a status bit, stops taking work and
+// leaves through the common exit (which frees its tensor memory).  A launch that finds the status
+// word set on entry does nothing.
 #pragma once
 
 #include <cuda.h>
