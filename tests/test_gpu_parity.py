@@ -126,6 +126,49 @@ def test_ragged_and_degenerate_blocks(dtype, path):
     _run(w, True, 8, path=path, blocks=_pack(RAGGED))
 
 
+ALIGNED_UNITS = [
+    # warp-sized units that start on 16-byte boundaries and hold a multiple of 8 elements ...
+    (40, 1600, A.MOM_NONE, 0, A.V_BLOCKMEAN, 1),        # one 1600-element row per unit, no momentum
+    (9, 2048, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1),         # units of the largest size
+    (300, 8, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1),          # units of the smallest size
+    (50, 1000, A.MOM_FULL, 0, A.V_ELEMENT, 0),          # per-element v, an 848-element tail unit
+    (3, 24, A.MOM_NONE, 0, A.V_ELEMENT, 0),             # one short unit
+    (1, 2040, A.MOM_FULL, 0, A.V_BLOCKMEAN, 0),         # whole-block group in one unit
+    (6000, 64, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1),        # many more units than CTAs
+    # ... next to blocks whose units are not
+    (33, 5, A.MOM_NONE, 0, A.V_BLOCKMEAN, 1),
+    (12, 1000, A.MOM_FULL, 0, A.V_BLOCKMEAN, 4),
+    (100, 77, A.MOM_FULL, 0, A.V_ELEMENT, 0),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_streaming_update_unit_shapes(dtype):
+    """Blocks without low-rank momentum over the unit shapes the streaming kernel distinguishes (vector and
+    guarded chunks, one or several batches per thread, with and without m and per-element v): all blocks against
+    the oracle, every step."""
+    w = WL.Workload("aligned_units", [], dtype, "normal", steps=6)
+    _run(w, True, 6, blocks=_pack(ALIGNED_UNITS))
+
+
+def test_streaming_update_with_clipping_and_shadow():
+    """The same blocks with the gradients scaled by the global clip factor and the bf16 copy of W written."""
+    import torch
+    w = WL.Workload("aligned_units", [], "bf16", "normal", steps=4)
+    run = ParityRun(w, True, custom_blocks=_pack(ALIGNED_UNITS), hp_overrides=dict(max_grad_norm=0.5), shadow=True)
+    try:
+        for _ in range(4):
+            run.step()
+            run.compare()
+            # padding between blocks is never written: compare the blocks' own ranges
+            for blk in run.blocks:
+                sl = slice(blk.offset, blk.offset + blk.rows * blk.cols)
+                assert torch.equal(run.shadow[sl], run.params[sl].to(torch.bfloat16))
+        assert run.ctx.adapm_get_status() == 0
+    finally:
+        run.close()
+
+
 def test_adam_debias_and_no_clip():
     w = WL.Workload("debias", [], "f32", "normal", steps=6)
     _run(w, True, 6, blocks=_pack(RAGGED[:8]), hp=dict(adam_debias=1, clip=math.inf))
