@@ -41,6 +41,11 @@ Readings of the paper taken here (each is a choice; the paper does not settle it
     T = 1 is Algorithm 1 as printed.  The function itself is pinned to the mathematics (tests): T = 1 equals
     the default, held-L passes equal scalar loops, and with orthonormal L and step size 1 one pass lands on
     the least-squares R = L^T m_t.
+  * A data-driven L_0 (`init_L0_range`; not in the paper, PARITY UNPINNED against it): instead of Gaussian
+    draws, L_0 spans what the first gradient spans.  With Omega an n x r Gaussian matrix handed in by the caller,
+    L_0 = the columns of g_1 Omega orthonormalised by modified Gram-Schmidt, in order, rounded to fp32 (the
+    randomized range finder); R_0 = 0 as before.  A column whose remainder after the projections has less than
+    1e-8 of its squared length left (g_1 has rank below r) becomes zero and stays zero under Algorithm 2.
 Parity with the authors' unreleased code on these readings is unpinned; what is
 pinned (tests/test_oracle_pins.py) is this oracle against closed forms, special
 cases, a library optimizer, the proof identity of Theorem 2 and brute force.
@@ -147,6 +152,26 @@ def init_L0(rows: int, rank: int, seed: int, block_index: int) -> np.ndarray:
         for i in range(j):
             q -= (Q[:, i] @ q) * Q[:, i]
         Q[:, j] = q / math.sqrt(q @ q)
+    return Q.astype(np.float32).astype(np.float64)
+
+
+RANGE_DROP = 1e-8     # a column of g Omega that keeps less than this share of its squared length is dropped
+
+
+def init_L0_range(g: np.ndarray, omega: np.ndarray) -> np.ndarray:
+    """Data-driven L_0: modified Gram-Schmidt over the columns of Y = g Omega, in order (randomized range finder).
+    g: [rows, cols], omega: [cols, rank].  Returns [rows, rank] with orthonormal (or zero) columns, rounded to fp32."""
+    Y = np.asarray(g, dtype=np.float64) @ np.asarray(omega, dtype=np.float64)
+    rows, rank = Y.shape
+    Q = np.zeros_like(Y)
+    for j in range(rank):
+        q = Y[:, j].copy()
+        n0 = q @ q
+        for i in range(j):
+            q -= (Q[:, i] @ q) * Q[:, i]
+        n1 = q @ q
+        if n0 > 0.0 and n1 > RANGE_DROP * n0:
+            Q[:, j] = q / math.sqrt(n1)
     return Q.astype(np.float32).astype(np.float64)
 
 

@@ -568,3 +568,55 @@ def test_held_L_passes_equal_scalar_loops_and_hit_least_squares_with_orthonormal
     eta1 = 0.5 * (1.0 + math.cos(math.pi / 2))
     _, R1 = O.lowrank_refit_gd(tgt, Q, RNG.standard_normal((3, 5)), 2, 1.0 / eta1, update_L=False)
     np.testing.assert_allclose(R1, Q.T @ tgt, rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------------------------------------------
+# Data-driven L_0 (randomized range finder on the first gradient; not in the paper)
+# ------------------------------------------------------------------------------------------------
+
+def test_range_L0_is_orthonormal_and_equals_qr_up_to_column_signs():
+    rng = np.random.default_rng(11)
+    g = rng.standard_normal((60, 45)); om = rng.standard_normal((45, 7))
+    L0 = O.init_L0_range(g, om)
+    assert np.array_equal(L0, L0.astype(np.float32).astype(np.float64))
+    assert np.abs(L0.T @ L0 - np.eye(7)).max() < 5e-7
+    # Gram-Schmidt in column order is the thin QR factorisation with a positive diagonal
+    Q, Rq = np.linalg.qr(g @ om)
+    Q = Q * np.sign(np.diag(Rq))
+    assert np.abs(L0 - Q).max() < 5e-7
+
+
+def test_range_L0_spans_the_range_of_a_rank_r_gradient_whatever_omega_is():
+    rng = np.random.default_rng(12)
+    U, _ = np.linalg.qr(rng.standard_normal((50, 4)))
+    g = U @ np.diag([3.0, 2.0, 1.0, 0.5]) @ rng.standard_normal((4, 30))
+    P = U @ U.T
+    for seed in (1, 2):
+        L0 = O.init_L0_range(g, np.random.default_rng(seed).standard_normal((30, 4)))
+        assert np.abs(L0 @ L0.T - P).max() < 1e-6          # the projector is unique, the basis is not
+    # more columns than the gradient has rank: the first four span it, the rest are dropped (zero)
+    L0 = O.init_L0_range(g, rng.standard_normal((30, 6)))
+    assert np.abs(L0[:, :4] @ L0[:, :4].T - P).max() < 1e-6
+    assert np.all(L0[:, 4:] == 0.0)
+
+
+def test_range_L0_of_a_rank_one_gradient_and_of_a_zero_gradient():
+    rng = np.random.default_rng(13)
+    u = rng.standard_normal(20); v = rng.standard_normal(9)
+    om = rng.standard_normal((9, 3))
+    L0 = O.init_L0_range(np.outer(u, v), om)
+    s = np.sign((v @ om)[0])
+    assert np.abs(L0[:, 0] - s * u / np.linalg.norm(u)).max() < 1e-7
+    assert np.all(L0[:, 1:] == 0.0)
+    assert np.all(O.init_L0_range(np.zeros((20, 9)), om) == 0.0)
+
+
+def test_a_dropped_column_of_L0_never_leaves_zero():
+    """Algorithm 2 from (L_0, R_0 = 0) with a zero column j in L_0: row j of dl/dR is L[:, j]^T E = 0 and column j of
+    dl/dL is E R[j, :]^T = 0, so the pair stays zero: the block simply runs at a lower rank."""
+    rng = np.random.default_rng(14)
+    g = np.outer(rng.standard_normal(12), rng.standard_normal(8))
+    L0 = O.init_L0_range(g, rng.standard_normal((8, 3)))
+    L, R = O.lowrank_refit_gd(0.1 * g + 0.01 * rng.standard_normal((12, 8)), L0, np.zeros((3, 8)), 5)
+    assert np.all(L[:, 1:] == 0.0) and np.all(R[1:, :] == 0.0)
+    assert np.abs(R[0]).max() > 0.0
