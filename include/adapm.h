@@ -167,6 +167,23 @@ int adapm_set_workspace(adapm_ctx* ctx, void* dev_ptr, size_t bytes);
  */
 int adapm_state_init(adapm_ctx* ctx, void* state, adapm_stream stream);
 
+/*
+ * Data-driven start (a variant; the paper gives none): zero the state and give every low-rank block
+ * L_0 = the columns of g_1 Omega orthonormalised in order by Gram-Schmidt (the randomized range finder),
+ * so that L_0 spans what the first gradient spans; R_0 = 0.  A column that keeps less than 1e-8 of its
+ * squared length (g_1 has rank below r) becomes zero and the block runs at a lower rank.
+ *   grads: device, the first step's gradients, same layout and dtype as for adapm_step (16-B aligned);
+ *   omega: device, fp32, adapm_init_omega_floats() floats, 16-B aligned, owned by the caller and only
+ *          read: block b's Omega is [cols, rank] row-major at the offset adapm_init_omega_layout
+ *          returns (count 0 for blocks without low-rank momentum).  The caller draws it (standard
+ *          normal entries): the library draws nothing here.
+ * Asynchronous on `stream`.  Errors: ADAPM_EINVAL (null pointers), ADAPM_EALIGN, ADAPM_ECUDA.
+ */
+int64_t adapm_init_omega_floats(const adapm_ctx* ctx);
+int adapm_init_omega_layout(const adapm_ctx* ctx, int64_t block, int64_t* offset, int64_t* count);
+int adapm_state_init_from_grads(adapm_ctx* ctx, void* state, const void* grads, const float* omega,
+                                adapm_stream stream);
+
 /* Learning rate eta_t of the next steps (Algorithm 1 takes a schedule; the caller owns it). */
 int adapm_set_lr(adapm_ctx* ctx, float lr);
 

@@ -27,6 +27,7 @@ EXPORTS = (
     "adapm_step_bytes", "adapm_step_flops", "adapm_launch_count", "adapm_get_status",
     "adapm_group_meansq_scratch_bytes", "adapm_group_meansq", "adapm_set_profiling", "adapm_get_launch_times",
     "adapm_launch_kind_name", "adapm_group_meansq_static", "adapm_state_changed", "adapm_selftest_expired_wait", "adapm_set_shadow_params",
+    "adapm_init_omega_floats", "adapm_init_omega_layout", "adapm_state_init_from_grads",
 )
 
 
@@ -117,6 +118,9 @@ def load(build_if_missing: bool = True) -> C.CDLL:
         "adapm_state_changed": (C.c_int, [vp]),
         "adapm_selftest_expired_wait": (C.c_int, [vp, vp]),
         "adapm_set_shadow_params": (C.c_int, [vp, vp]),
+        "adapm_init_omega_floats": (i64, [vp]),
+        "adapm_init_omega_layout": (C.c_int, [vp, i64, C.POINTER(i64), C.POINTER(i64)]),
+        "adapm_state_init_from_grads": (C.c_int, [vp, vp, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -227,6 +231,18 @@ class Context:
 
     def adapm_state_init(self, state, stream=None) -> None:
         _check(self._lib.adapm_state_init(self._h, _ptr(state), _stream(stream)), "adapm_state_init")
+
+    def adapm_init_omega_floats(self) -> int:
+        return self._lib.adapm_init_omega_floats(self._h)
+
+    def adapm_init_omega_layout(self, block: int) -> Tuple[int, int]:
+        off, cnt = C.c_int64(), C.c_int64()
+        _check(self._lib.adapm_init_omega_layout(self._h, block, C.byref(off), C.byref(cnt)), "adapm_init_omega_layout")
+        return off.value, cnt.value
+
+    def adapm_state_init_from_grads(self, state, grads, omega, stream=None) -> None:
+        _check(self._lib.adapm_state_init_from_grads(self._h, _ptr(state), _ptr(grads), _ptr(omega), _stream(stream)),
+               "adapm_state_init_from_grads")
 
     def adapm_set_lr(self, lr: float) -> None:
         _check(self._lib.adapm_set_lr(self._h, lr), "adapm_set_lr")

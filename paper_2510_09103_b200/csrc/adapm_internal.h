@@ -178,7 +178,7 @@ int launch_meansq_partial(const void* g, int grad_dtype, int64_t n_groups, int64
                           float* partial, cudaStream_t s);
 int launch_meansq_final(const float* partial, int64_t n_groups, int64_t group_elems, int chunks_per_group, float* out,
                         cudaStream_t s);
-int launch_init_L0(const InitJob* d_tab, int64_t n_jobs, float* state, uint64_t seed, cudaStream_t s);
+int launch_init_L0(const InitJob* d_tab, int64_t n_jobs, float* state, uint64_t seed, int draw, cudaStream_t s);
 
 struct TcProgram;   // host side of the tensor-core low-rank path (lowrank_tc.cu)
 
@@ -208,6 +208,10 @@ struct adapm_ctx {
   unsigned char* d_tables = nullptr;
   int32_t* d_status = nullptr;
   int64_t init_table_off = 0, n_init_jobs = 0;
+  // data-driven L_0: Y = g Omega per low-rank block (one batched GEMM), Omega in a caller buffer laid out by omega_off
+  std::vector<int64_t> omega_off;      // float offset of a block's Omega [cols, rank], -1 for other blocks
+  int64_t omega_floats = 0;
+  int64_t range_table_off = 0, n_range_probs = 0, n_range_tiles = 0;
   int final_lr_buf = -1;               // which workspace copy holds L_t,R_t after the refit (-1: unchanged)
   adapm::TcProgram* tc = nullptr;      // program of the blocks that run on the tensor cores
   int64_t n_tensor_blocks = 0;

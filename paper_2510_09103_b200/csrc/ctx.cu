@@ -290,6 +290,30 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         ijobs.push_back({c->l_off[i], i, c->blocks[i].rows, c->blocks[i].rank});
     c->init_table_off = append_table(c->h_tables, ijobs);
     c->n_init_jobs = (int64_t)ijobs.size();
+    // Y = g Omega -> the block's L in the state (data-driven L_0)
+    c->omega_off.assign(n, -1);
+    std::vector<GemmProb> rp;
+    int64_t tiles = 0;
+    for (int pass = 0; pass < 2; ++pass)
+      for (int64_t i : (pass == 0 ? lowrank_ids : tc_ids)) {
+        const adapm_block& b = c->blocks[i];
+        c->omega_off[i] = c->omega_floats;
+        c->omega_floats += round_up((int64_t)b.cols * b.rank, kStateAlign);
+        GemmProb p;
+        std::memset(&p, 0, sizeof(p));
+        p.z1_base = p.z2_base = BASE_NONE;
+        p.alpha = 1.f;
+        p.x_base = BASE_GRADS; p.x_off = b.offset; p.sxi = b.cols; p.sxk = 1;
+        p.y_base = BASE_WORK; p.y_off = c->omega_off[i]; p.syk = b.rank; p.syj = 1;
+        p.c_base = BASE_STATE; p.c_off = c->l_off[i]; p.M = b.rows; p.N = b.rank; p.K = b.cols; p.ldc = b.rank;
+        p.tiles_n = (p.N + 63) / 64;
+        p.first_tile = tiles;
+        tiles += (int64_t)((p.M + 63) / 64) * p.tiles_n;
+        rp.push_back(p);
+      }
+    c->range_table_off = append_table(c->h_tables, rp);
+    c->n_range_probs = (int64_t)rp.size();
+    c->n_range_tiles = tiles;
   }
   if (!tc_ids.empty()) {
     std::vector<ReduceJob> row_jobs;
@@ -521,8 +545,38 @@ extern "C" int adapm_state_init(adapm_ctx* c, void* state, adapm_stream stream) 
   ADAPM_CUDA(cudaMemsetAsync(state, 0, (size_t)c->state_floats * 4, s));
   tensor_state_changed(c);
   if (c->n_init_jobs > 0)
-    return launch_init_L0((const InitJob*)(c->d_tables + c->init_table_off), c->n_init_jobs, (float*)state, c->hp.seed, s);
+    return launch_init_L0((const InitJob*)(c->d_tables + c->init_table_off), c->n_init_jobs, (float*)state, c->hp.seed, 1, s);
   return ADAPM_OK;
+}
+
+extern "C" int64_t adapm_init_omega_floats(const adapm_ctx* c) { return c ? c->omega_floats : 0; }
+
+extern "C" int adapm_init_omega_layout(const adapm_ctx* c, int64_t block, int64_t* offset, int64_t* count) {
+  if (!c || !offset || !count) return ADAPM_EINVAL;
+  if (block < 0 || block >= (int64_t)c->blocks.size()) return ADAPM_ERANGE;
+  const bool lowrank = !c->omega_off.empty() && c->omega_off[(size_t)block] >= 0;
+  *offset = lowrank ? c->omega_off[(size_t)block] : 0;
+  *count = lowrank ? (int64_t)c->blocks[(size_t)block].cols * c->blocks[(size_t)block].rank : 0;
+  return ADAPM_OK;
+}
+
+extern "C" int adapm_state_init_from_grads(adapm_ctx* c, void* state, const void* grads, const float* omega,
+                                           adapm_stream stream) {
+  if (!c || !state || !grads) return ADAPM_EINVAL;
+  if (c->n_init_jobs > 0 && !omega) return ADAPM_EINVAL;
+  if ((uintptr_t)state % 256 || (uintptr_t)grads % 16 || (uintptr_t)omega % 16) return ADAPM_EALIGN;
+  cudaStream_t s = (cudaStream_t)stream;
+  ADAPM_CUDA(cudaMemsetAsync(state, 0, (size_t)c->state_floats * 4, s));
+  tensor_state_changed(c);
+  if (c->n_init_jobs == 0) return ADAPM_OK;
+  Bases b;
+  b.p[BASE_PARAMS] = nullptr; b.p[BASE_GRADS] = const_cast<void*>(grads); b.p[BASE_STATE] = state;
+  b.p[BASE_WORK] = const_cast<float*>(omega);
+  b.status = c->d_status; b.gscale = nullptr; b.shadow = nullptr;
+  const int rc = launch_gemm((const GemmProb*)(c->d_tables + c->range_table_off), c->n_range_probs, c->n_range_tiles, b,
+                             c->hp.grad_dtype, s);
+  if (rc != ADAPM_OK) return rc;
+  return launch_init_L0((const InitJob*)(c->d_tables + c->init_table_off), c->n_init_jobs, (float*)state, c->hp.seed, 0, s);
 }
 
 extern "C" int adapm_set_lr(adapm_ctx* c, float lr) {

@@ -201,17 +201,31 @@ __device__ __forceinline__ float block_sum_1024(float x, float* red) {
   return s;
 }
 
+// Modified Gram-Schmidt over the columns of L, in order, one CTA per block.  draw = 1: the columns are Gaussian
+// draws first (keyed by seed, block, element).  draw = 0: L already holds the matrix to orthonormalise (g Omega of
+// the data-driven start); a column that keeps less than kRangeDrop of its squared length becomes zero.
+constexpr float kRangeDrop = 1e-8f;
+
 __global__ void __launch_bounds__(1024) init_L0_kernel(const InitJob* __restrict__ tab, float* __restrict__ state,
-                                                       uint64_t seed) {
+                                                       uint64_t seed, int draw) {
   __shared__ float red[32];
   const InitJob J = tab[blockIdx.x];
   float* __restrict__ L = state + J.l_off;
   const int rows = J.rows, rank = J.rank;
   const uint64_t block = (uint64_t)J.block_index;
   const int64_t total = (int64_t)rows * rank;
-  for (int64_t e = threadIdx.x; e < total; e += blockDim.x) L[e] = gaussian_from_counter(seed, block, (uint64_t)e);
+  if (draw)
+    for (int64_t e = threadIdx.x; e < total; e += blockDim.x) L[e] = gaussian_from_counter(seed, block, (uint64_t)e);
   __syncthreads();
   for (int j = 0; j < rank; ++j) {
+    float n0 = 0.f;
+    if (!draw) {
+      for (int row = threadIdx.x; row < rows; row += blockDim.x) {
+        const float x = L[(int64_t)row * rank + j];
+        n0 += x * x;
+      }
+      n0 = block_sum_1024(n0, red);
+    }
     for (int i = 0; i < j; ++i) {
       float d = 0.f;
       for (int row = threadIdx.x; row < rows; row += blockDim.x) d += L[(int64_t)row * rank + i] * L[(int64_t)row * rank + j];
@@ -224,7 +238,7 @@ __global__ void __launch_bounds__(1024) init_L0_kernel(const InitJob* __restrict
       nn += x * x;
     }
     nn = block_sum_1024(nn, red);
-    const float inv = rsqrtf(nn);
+    const float inv = (draw || (n0 > 0.f && nn > kRangeDrop * n0)) ? rsqrtf(nn) : 0.f;
     for (int row = threadIdx.x; row < rows; row += blockDim.x) L[(int64_t)row * rank + j] *= inv;
     __syncthreads();
   }
@@ -263,9 +277,9 @@ int launch_apply_simt(const ApplyBlk* d_tab, int64_t n_blk, int64_t n_tiles, con
   return ADAPM_OK;
 }
 
-int launch_init_L0(const InitJob* d_tab, int64_t n_jobs, float* state, uint64_t seed, cudaStream_t s) {
+int launch_init_L0(const InitJob* d_tab, int64_t n_jobs, float* state, uint64_t seed, int draw, cudaStream_t s) {
   if (n_jobs <= 0) return ADAPM_OK;
-  init_L0_kernel<<<(unsigned)n_jobs, 1024, 0, s>>>(d_tab, state, seed);
+  init_L0_kernel<<<(unsigned)n_jobs, 1024, 0, s>>>(d_tab, state, seed, draw);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }

@@ -204,6 +204,106 @@ def test_state_init_gives_orthonormal_L0_and_zero_R0():
     ctx.adapm_destroy()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_state_init_from_grads_matches_the_range_finder_oracle(dtype):
+    """Data-driven L_0 = Gram-Schmidt over the columns of g_1 Omega (a variant, not in the paper): the library's L_0
+    against the oracle's, element by element; a gradient of rank 2 under rank 5 leaves three zero columns on both
+    sides; R, v and the other blocks' state are zero."""
+    import torch
+    specs = [(300, 64, A.MOM_LOWRANK, 12, A.V_BLOCKMEAN, 1), (64, 504, A.MOM_LOWRANK, 5, A.V_ELEMENT, 0),
+             (40, 16, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1), (640, 384, A.MOM_LOWRANK, 38, A.V_BLOCKMEAN, 1),
+             (96, 72, A.MOM_LOWRANK, 5, A.V_BLOCKMEAN, 1)]
+    blocks = _pack(specs)
+    total = -(-max(b.offset + b.rows * b.cols for b in blocks) // 8) * 8
+    rng = np.random.default_rng(5)
+    g = np.zeros(total, dtype=np.float32)
+    for bi, b in enumerate(blocks):
+        x = rng.standard_normal((b.rows, b.cols)) * 1e-3 * np.exp(rng.uniform(-2, 2, size=(b.rows, 1)))
+        if bi == 4:     # rank 2, small integers times 2^-10: exact in bf16, so rounding does not fill the rank up
+            x = (rng.integers(-3, 4, size=(b.rows, 2)) @ rng.integers(-3, 4, size=(2, b.cols))) * 2.0 ** -10
+        g[b.offset:b.offset + b.rows * b.cols] = x.ravel()
+    if dtype == "bf16":
+        gt = torch.from_numpy(g).to(torch.bfloat16)
+        g = gt.to(torch.float32).numpy()
+    else:
+        gt = torch.from_numpy(g)
+    ctx = A.adapm_create(blocks, A.hparams(grad_dtype=A.GRAD_BF16 if dtype == "bf16" else A.GRAD_F32))
+    omega = np.zeros(ctx.adapm_init_omega_floats(), dtype=np.float32)
+    om_of = {}
+    for bi, b in enumerate(blocks):
+        off, cnt = ctx.adapm_init_omega_layout(bi)
+        assert cnt == (b.cols * b.rank if b.mom_mode == A.MOM_LOWRANK else 0)
+        if cnt:
+            om_of[bi] = rng.standard_normal((b.cols, b.rank)).astype(np.float32)
+            omega[off:off + cnt] = om_of[bi].ravel()
+    state = torch.full((ctx.adapm_state_bytes() // 4,), 3.0, device="cuda")
+    ctx.adapm_state_init_from_grads(state, gt.cuda(), torch.from_numpy(omega).cuda())
+    torch.cuda.synchronize()
+    host = state.cpu().numpy()
+    seen = np.zeros(host.size, dtype=bool)
+    for bi, b in enumerate(blocks):
+        if b.mom_mode != A.MOM_LOWRANK:
+            continue
+        off, cnt = ctx.adapm_state_layout(bi, A.STATE_L)
+        L = host[off:off + cnt].reshape(b.rows, b.rank).astype(np.float64)
+        seen[off:off + cnt] = True
+        ref = O.init_L0_range(g[b.offset:b.offset + b.rows * b.cols].reshape(b.rows, b.cols).astype(np.float64),
+                              om_of[bi].astype(np.float64))
+        assert rel_err(L, ref) <= 1e-4, (bi, rel_err(L, ref))
+        if bi == 4:
+            assert np.all(L[:, 2:] == 0.0) and np.all(ref[:, 2:] == 0.0)
+            np.testing.assert_allclose(L[:, :2].T @ L[:, :2], np.eye(2), atol=2e-5)
+        else:
+            np.testing.assert_allclose(L.T @ L, np.eye(b.rank), atol=5e-5)
+    assert not host[~seen].any()            # R_0, v, m and the padding: all zero
+    assert ctx.adapm_get_status() == 0
+    ctx.adapm_destroy()
+
+
+def test_steps_from_a_data_driven_L0_follow_the_oracle():
+    """Three steps started from the library's own range-finder L_0 (handed to the oracle as its L_0), on the CUDA-core
+    and on the tensor-core refit."""
+    import torch
+    for path, dtype in ((A.PATH_SIMT, "f32"), (A.PATH_TENSOR, "bf16")):
+        blocks = _pack([(256, 192, A.MOM_LOWRANK, 38, A.V_BLOCKMEAN, 1), (384, 128, A.MOM_LOWRANK, 16, A.V_BLOCKMEAN, 1),
+                        (64, 512, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1)])
+        run = ParityRun(WL.Workload("range_start", [], dtype, "normal", steps=3), True, lowrank_path=path,
+                        custom_blocks=blocks)
+        try:
+            # the first step's gradients, as the harness will hand them to the step
+            np_dt = np.uint16 if dtype == "bf16" else np.float32
+            host = np.zeros(run.total, dtype=np_dt)
+            for ti in range(len(run.w.tensors)):
+                _, raw = run._grad_raw(ti, 1)
+                off = run.blocks[run.t2b[ti][0]].offset
+                host[off:off + raw.size] = raw
+            g1 = torch.from_numpy(host.view(np.int16) if dtype == "bf16" else host).cuda()
+            g1 = g1.view(torch.bfloat16) if dtype == "bf16" else g1
+            rng = np.random.default_rng(9)
+            omega = torch.from_numpy(rng.standard_normal(run.ctx.adapm_init_omega_floats()).astype(np.float32)).cuda()
+            canary_state = run.state.clone()
+            run.ctx.adapm_state_init_from_grads(run.state, g1, omega)
+            torch.cuda.synchronize()
+            # keep the harness's canaries in the gaps of the state buffer; take the new sub-buffers
+            fresh = run.state.clone()
+            run.state.copy_(canary_state)
+            for bi, b in enumerate(run.blocks):
+                for which in (A.STATE_M, A.STATE_L, A.STATE_R, A.STATE_V):
+                    off, cnt = run.ctx.adapm_state_layout(bi, which)
+                    if cnt:
+                        run.state[off:off + cnt] = fresh[off:off + cnt]
+                if b.mom_mode == A.MOM_LOWRANK:
+                    off, cnt = run.ctx.adapm_state_layout(bi, A.STATE_L)
+                    run.ostate[bi].L = run.state[off:off + cnt].cpu().numpy().reshape(b.rows, b.rank).astype(np.float64)
+            run.ctx.adapm_state_changed()
+            for _ in range(3):
+                run.step()
+                run.compare()
+            assert run.ctx.adapm_get_status() == 0
+        finally:
+            run.close()
+
+
 def test_runs_are_bitwise_reproducible_and_resumable():
     import torch
     w = WL.get_workload("tiny")
