@@ -46,6 +46,10 @@ Readings of the paper taken here (each is a choice; the paper does not settle it
     L_0 = the columns of g_1 Omega orthonormalised by modified Gram-Schmidt, in order, rounded to fp32 (the
     randomized range finder); R_0 = 0 as before.  A column whose remainder after the projections has less than
     1e-8 of its squared length left (g_1 has rank below r) becomes zero and stays zero under Algorithm 2.
+  * Preconditioned inner passes (`inner_precond`, `lowrank_refit_scaled_gd`; not in the paper, PARITY UNPINNED
+    against it): each derivative of Algorithm 2 is multiplied by the damped inverse of the other factor's Gram
+    matrix (scaled gradient descent), which makes the pass independent of how the product L R is split between
+    the factors; everything else of Algorithm 2 (warm start, schedule, simultaneous update) is kept.
 Parity with the authors' unreleased code on these readings is unpinned; what is
 pinned (tests/test_oracle_pins.py) is this oracle against closed forms, special
 cases, a library optimizer, the proof identity of Theorem 2 and brute force.
@@ -98,6 +102,8 @@ class HParams:
     correction_off_uses_product: bool = False   # with correction off: m^c := L_t R_t instead of m_t
     max_grad_norm: float = math.inf   # global clipping threshold c; inf disables
     refresh_period: int = 1      # T: both factors are refitted at steps 1, T+1, 2T+1, ...; in between only R
+    inner_precond: bool = False  # preconditioned passes (ScaledGD) instead of Algorithm 2's plain ones
+    precond_damping: float = 1e-3     # delta = damping * trace(Gram) / r is added to the Gram matrix's diagonal
 
 
 @dataclass
@@ -130,6 +136,36 @@ def lowrank_refit_gd(m_t: np.ndarray, L_prev: np.ndarray, R_prev: np.ndarray, K:
         E = L @ R - m_t                  # L R - m_t
         dL = E @ R.T                     # dl/dL = (L R - m_t) R^T
         dR = L.T @ E                     # dl/dR = L^T (L R - m_t)
+        if update_L:
+            L = L - (scale * eta) * dL
+        R = R - (scale * eta) * dR
+    return L, R
+
+
+PRECOND_FLOOR = 1e-30    # keeps the damped Gram matrix invertible when the factor is exactly zero (R_0 = 0)
+
+
+def damped_inverse(G: np.ndarray, damping: float) -> np.ndarray:
+    """(G + delta I)^-1 with delta = damping * trace(G) / r + PRECOND_FLOOR, G a symmetric r x r Gram matrix."""
+    r = G.shape[0]
+    delta = damping * np.trace(G) / r + PRECOND_FLOOR
+    return np.linalg.inv(G + delta * np.eye(r))
+
+
+def lowrank_refit_scaled_gd(m_t: np.ndarray, L_prev: np.ndarray, R_prev: np.ndarray, K: int, scale: float = 1.0,
+                            damping: float = 1e-3, update_L: bool = True):
+    """Preconditioned passes in place of Algorithm 2's (a variant; not in the paper): the scaled gradient descent
+    of Tong, Ma and Chi (2021) for low-rank factorisation, with a damped preconditioner,
+        L <- L - eta_k (L R - m_t) R^T (R R^T + delta_R I)^-1,   R <- R - eta_k (L^T L + delta_L I)^-1 L^T (L R - m_t),
+    both from the same point, same schedule and warm start as Algorithm 2."""
+    L = np.array(L_prev, dtype=np.float64, copy=True)
+    R = np.array(R_prev, dtype=np.float64, copy=True)
+    if K <= 0:
+        return L, R
+    for eta in inner_schedule(K):
+        E = L @ R - m_t
+        dL = (E @ R.T) @ damped_inverse(R @ R.T, damping)
+        dR = damped_inverse(L.T @ L, damping) @ (L.T @ E)
         if update_L:
             L = L - (scale * eta) * dL
         R = R - (scale * eta) * dR
@@ -251,7 +287,11 @@ def block_step(W: np.ndarray, g: np.ndarray, st: BlockState, blk: Block, hp: HPa
         m_t = (1.0 - b1) * g + b1 * P_prev                     # line 4
         if solver == "gd":
             refresh = hp.refresh_period <= 1 or (t - 1) % hp.refresh_period == 0
-            L, R = lowrank_refit_gd(m_t, st.L, st.R, hp.inner_iters, hp.inner_lr_scale, update_L=refresh)   # line 5
+            if hp.inner_precond:
+                L, R = lowrank_refit_scaled_gd(m_t, st.L, st.R, hp.inner_iters, hp.inner_lr_scale, hp.precond_damping,
+                                               update_L=refresh)
+            else:
+                L, R = lowrank_refit_gd(m_t, st.L, st.R, hp.inner_iters, hp.inner_lr_scale, update_L=refresh)   # line 5
         elif solver == "exact":
             L, R = lowrank_refit_exact(m_t, blk.rank)
         else:

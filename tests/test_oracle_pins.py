@@ -620,3 +620,87 @@ def test_a_dropped_column_of_L0_never_leaves_zero():
     L, R = O.lowrank_refit_gd(0.1 * g + 0.01 * rng.standard_normal((12, 8)), L0, np.zeros((3, 8)), 5)
     assert np.all(L[:, 1:] == 0.0) and np.all(R[1:, :] == 0.0)
     assert np.abs(R[0]).max() > 0.0
+
+
+# ------------------------------------------------------------------------------------------------
+# Preconditioned inner passes (scaled gradient descent; not in the paper)
+# ------------------------------------------------------------------------------------------------
+
+def _one_pass_schedule(monkeypatch, etas):
+    monkeypatch.setattr(O, "inner_schedule", lambda K: list(etas))
+
+
+def test_scaled_gd_full_step_lands_on_the_two_least_squares_solutions(monkeypatch):
+    """One pass with step size 1 and no damping: R' = argmin_R ||L R - m|| and L' = argmin_L ||L R - m||, each with
+    the other factor at its old value (both derivatives are taken at the same point)."""
+    rng = np.random.default_rng(21)
+    m = rng.standard_normal((9, 7)); L = rng.standard_normal((9, 3)); R = rng.standard_normal((3, 7))
+    _one_pass_schedule(monkeypatch, [1.0])
+    L1, R1 = O.lowrank_refit_scaled_gd(m, L, R, 1, damping=0.0)
+    np.testing.assert_allclose(R1, np.linalg.lstsq(L, m, rcond=None)[0], atol=1e-10)
+    np.testing.assert_allclose(L1, np.linalg.lstsq(R.T, m.T, rcond=None)[0].T, atol=1e-10)
+
+
+def test_scaled_gd_does_not_depend_on_how_the_product_is_split():
+    """(L, R) -> (L Q, Q^-1 R) leaves L R unchanged; without damping the preconditioned passes then produce the same
+    product again (plain gradient descent does not)."""
+    rng = np.random.default_rng(22)
+    m = rng.standard_normal((10, 8)); L = rng.standard_normal((10, 3)); R = rng.standard_normal((3, 8))
+    Q = rng.standard_normal((3, 3)) + 3 * np.eye(3)
+    La, Ra = O.lowrank_refit_scaled_gd(m, L, R, 5, scale=0.5, damping=0.0)
+    Lb, Rb = O.lowrank_refit_scaled_gd(m, L @ Q, np.linalg.inv(Q) @ R, 5, scale=0.5, damping=0.0)
+    np.testing.assert_allclose(La @ Ra, Lb @ Rb, atol=1e-9)
+    Lc, Rc = O.lowrank_refit_gd(m, L @ Q, np.linalg.inv(Q) @ R, 5, 0.01)
+    Ld, Rd = O.lowrank_refit_gd(m, L, R, 5, 0.01)
+    assert np.abs(Lc @ Rc - Ld @ Rd).max() > 1e-4
+
+
+def test_scaled_gd_rank_one_equals_scalar_loops():
+    rng = np.random.default_rng(23)
+    m = rng.standard_normal((3, 2)); L = rng.standard_normal((3, 1)); R = rng.standard_normal((1, 2))
+    damping = 0.05
+    l = [float(x) for x in L[:, 0]]; r = [float(x) for x in R[0]]
+    for eta in O.inner_schedule(5):
+        rr = sum(x * x for x in r); ll = sum(x * x for x in l)
+        sr = 1.0 / (rr + damping * rr + O.PRECOND_FLOOR); sl = 1.0 / (ll + damping * ll + O.PRECOND_FLOOR)
+        e = [[l[i] * r[j] - m[i, j] for j in range(2)] for i in range(3)]
+        dl = [sum(e[i][j] * r[j] for j in range(2)) * sr for i in range(3)]
+        dr = [sum(l[i] * e[i][j] for i in range(3)) * sl for j in range(2)]
+        l = [l[i] - eta * dl[i] for i in range(3)]
+        r = [r[j] - eta * dr[j] for j in range(2)]
+    L5, R5 = O.lowrank_refit_scaled_gd(m, L, R, 5, damping=damping)
+    np.testing.assert_allclose(L5[:, 0], l, atol=1e-12)
+    np.testing.assert_allclose(R5[0], r, atol=1e-12)
+
+
+def test_scaled_gd_with_scalar_gram_matrices_is_plain_gd_with_rescaled_steps(monkeypatch):
+    """L with orthogonal columns of squared length d and R with orthogonal rows of squared length c: the
+    preconditioners are multiples of the identity, so one pass equals Algorithm 2's with the derivatives divided by
+    c (1 + damping) and d (1 + damping)."""
+    rng = np.random.default_rng(24)
+    QL, _ = np.linalg.qr(rng.standard_normal((8, 3))); QR, _ = np.linalg.qr(rng.standard_normal((6, 3)))
+    L = 2.0 * QL; R = 0.5 * QR.T
+    m = rng.standard_normal((8, 6))
+    _one_pass_schedule(monkeypatch, [0.4])
+    L1, R1 = O.lowrank_refit_scaled_gd(m, L, R, 1, damping=0.1)
+    E = L @ R - m
+    np.testing.assert_allclose(L1, L - 0.4 * (E @ R.T) / (0.25 * 1.1), atol=1e-12)
+    np.testing.assert_allclose(R1, R - 0.4 * (L.T @ E) / (4.0 * 1.1), atol=1e-12)
+
+
+def test_scaled_gd_from_R_zero_moves_R_only_and_block_step_uses_it():
+    rng = np.random.default_rng(25)
+    L0 = O.init_L0(12, 3, 0, 4); m = rng.standard_normal((12, 9)) * 1e-3
+    L1, R1 = O.lowrank_refit_scaled_gd(m, L0, np.zeros((3, 9)), 5)
+    assert np.all(np.isfinite(L1)) and np.all(np.isfinite(R1)) and np.abs(R1).max() > 0
+    blk = O.Block(rows=12, cols=9, mom_mode=O.MOM_LOWRANK, rank=3)
+    g = rng.standard_normal((12, 9)) * 1e-3
+    outs = []
+    for pre in (False, True):
+        st = O.new_state(blk, L0)
+        O.block_step(rng.standard_normal((12, 9)) * 0 + 0.01, g, st, blk, O.HParams(inner_precond=pre), 1)
+        outs.append((st.L.copy(), st.R.copy()))
+    Ls, Rs = O.lowrank_refit_scaled_gd(0.1 * g, L0, np.zeros((3, 9)), 5)
+    np.testing.assert_allclose(outs[1][0], Ls, atol=1e-14)
+    np.testing.assert_allclose(outs[1][1], Rs, atol=1e-14)
+    assert np.abs(outs[0][1] - outs[1][1]).max() > 0
