@@ -356,7 +356,7 @@ def run_gpu(args) -> None:
              | (A.FLAG_NO_SUMSQ_FOLD if args.no_fold else 0))
     hp = A.hparams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, grad_dtype=gd, lowrank_path=path, flags=flags,
                    tune_panels=args.panels, tune_stage_k=args.stage_k, max_grad_norm=args.max_grad_norm,
-                   refresh_period=args.refresh_period)
+                   refresh_period=args.refresh_period, inner_precond=1 if args.precond else 0)
     ctx = A.adapm_create(blocks, hp)
 
     # synthetic inputs: parameters N(0, 0.02^2) drawn on the device; gradients tiled from a seeded host pool
@@ -517,6 +517,7 @@ def run_gpu(args) -> None:
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "params": w.numel, "blocks": len(blocks), "v_mode": args.v_mode,
                    "max_grad_norm": args.max_grad_norm, "refresh_period": args.refresh_period, "bf16_shadow": args.shadow,
+                   "inner_precond": bool(args.precond),
                    "grad_dtype": w.grad_dtype, "state_dtype": "f32", "lowrank_path": args.path,
                    "lowrank_kernels": "tensor" if any(k.startswith("tc_") for k in kernels) else "simt",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
@@ -563,6 +564,8 @@ def main() -> None:
     ap.add_argument("--teams", default="auto", choices=["auto", "off", "force"], help="panel team schedule")
     ap.add_argument("--no-fold", action="store_true", help="row sums of g^2 from a pass of their own")
     ap.add_argument("--max-grad-norm", type=float, default=0.0, help="global gradient-norm clipping threshold (0 = off)")
+    ap.add_argument("--precond", action="store_true",
+                    help="preconditioned refit passes (a variant; CUDA-core path only)")
     ap.add_argument("--refresh-period", type=int, default=0, help="T: refit both factors every T steps (0/1 = every step)")
     ap.add_argument("--shadow", action="store_true", help="also write the bf16 copy of the parameters")
     args = ap.parse_args()

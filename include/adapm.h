@@ -116,6 +116,13 @@ typedef struct {
                               0 or 1 = Algorithm 1 as printed, every step                          */
   int32_t tune_panels;     /* tensor path: 128-row panels per refit item (1..3); 0 = automatic     */
   int32_t tune_stage_k;    /* tensor path: K per shared-memory stage (64 or 128); 0 = automatic    */
+  int32_t inner_precond;   /* 0 = Algorithm 2 as printed.  1 = preconditioned passes (a variant, not in
+                              the paper: scaled gradient descent): dl/dL is multiplied from the right
+                              by (R R^T + d_R I)^-1 and dl/dR from the left by (L^T L + d_L I)^-1, with
+                              d = precond_damping * trace / r + 1e-30; warm start, schedule and the
+                              simultaneous update are Algorithm 2's.  Runs on the CUDA-core path only
+                              (ADAPM_PATH_TENSOR with it: ADAPM_EUNSUPPORTED)                        */
+  float   precond_damping; /* >= 0; used when inner_precond = 1                                    */
 } adapm_hparams;
 
 /* Library version (major*100 + minor). */

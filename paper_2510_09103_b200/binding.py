@@ -54,15 +54,16 @@ class adapm_hparams(C.Structure):
                 ("grad_dtype", C.c_int32), ("adam_debias", C.c_int32), ("correction", C.c_int32),
                 ("lowrank_path", C.c_int32), ("seed", C.c_uint64), ("flags", C.c_uint32),
                 ("max_grad_norm", C.c_float), ("refresh_period", C.c_int32), ("tune_panels", C.c_int32),
-                ("tune_stage_k", C.c_int32)]
+                ("tune_stage_k", C.c_int32), ("inner_precond", C.c_int32), ("precond_damping", C.c_float)]
 
 
 def hparams(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, clip=1.0, inner_iters=5, inner_lr_scale=1.0,
             grad_dtype=GRAD_BF16, adam_debias=0, correction=1, lowrank_path=PATH_AUTO, seed=0, flags=0,
-            max_grad_norm=0.0, refresh_period=0, tune_panels=0, tune_stage_k=0) -> adapm_hparams:
+            max_grad_norm=0.0, refresh_period=0, tune_panels=0, tune_stage_k=0, inner_precond=0,
+            precond_damping=1e-3) -> adapm_hparams:
     return adapm_hparams(lr, beta1, beta2, eps, clip, inner_iters, inner_lr_scale, grad_dtype, adam_debias,
                          correction, lowrank_path, seed, flags, max_grad_norm, refresh_period, tune_panels,
-                         tune_stage_k)
+                         tune_stage_k, inner_precond, precond_damping)
 
 
 class AdapmError(RuntimeError):

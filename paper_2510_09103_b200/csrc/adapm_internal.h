@@ -117,6 +117,12 @@ struct ApplyBlk {
   int64_t first_tile;
 };
 
+// (G + delta I)^-1 of a symmetric r x r matrix, delta = damping * trace(G) / r + floor
+struct InverseJob {
+  int64_t src_off, dst_off;   // float offsets in the workspace
+  int32_t r, pad_;
+};
+
 struct InitJob {
   int64_t l_off;        // float offset of L in state
   int64_t block_index;  // keys the random stream
@@ -135,7 +141,8 @@ enum LaunchKind : int32_t {
   LK_TC_CONVERT, LK_TC_GRAM, LK_TC_PANEL, LK_TC_APPLY,
   LK_REDUCE_ROWS,       // reduce_final over the row sums of g^2 that the first refit pass left
   LK_GRADNORM,          // global gradient norm and the clip factor
-  LK_TC_COPY            // previous split copy of L -> final set (steps that hold L)
+  LK_TC_COPY,           // previous split copy of L -> final set (steps that hold L)
+  LK_SPD_INVERSE        // damped inverses of the r x r Gram matrices (preconditioned passes)
 };
 // when a launch of the program runs
 enum LaunchWhen : int32_t {
@@ -172,6 +179,8 @@ int launch_gemm(const GemmProb* d_tab, int64_t n_prob, int64_t n_tiles, const Ba
                 cudaStream_t s);
 int launch_apply_simt(const ApplyBlk* d_tab, int64_t n_blk, int64_t n_tiles, const Bases& b, const StepScalars& sc,
                       int grad_dtype, cudaStream_t s);
+int launch_spd_inverse(const InverseJob* d_tab, int64_t n_jobs, float* work, float damping, const int32_t* status,
+                       cudaStream_t s);
 int launch_copy_ranges(const NormRange* d_tab, const int32_t* d_cta_range, int64_t n_ctas, float* dst, const float* src,
                        const int32_t* status, cudaStream_t s);
 int launch_meansq_partial(const void* g, int grad_dtype, int64_t n_groups, int64_t group_elems, int chunks_per_group,

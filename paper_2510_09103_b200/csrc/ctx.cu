@@ -42,6 +42,8 @@ int validate(const adapm_block* blocks, int64_t n, const adapm_hparams& hp) {
   if (!(hp.max_grad_norm >= 0.f)) return ADAPM_ERANGE;      // 0 and +inf both mean "no clipping"; NaN is refused
   if (hp.tune_panels < 0 || hp.tune_panels > 3) return ADAPM_ERANGE;
   if (hp.tune_stage_k != 0 && hp.tune_stage_k != 64 && hp.tune_stage_k != 128) return ADAPM_ERANGE;
+  if (hp.inner_precond != 0 && hp.inner_precond != 1) return ADAPM_EINVAL;
+  if (hp.inner_precond && !(hp.precond_damping >= 0.f && std::isfinite(hp.precond_damping))) return ADAPM_ERANGE;
   std::vector<std::pair<int64_t, int64_t>> spans;
   spans.reserve((size_t)n);
   for (int64_t i = 0; i < n; ++i) {
@@ -106,8 +108,10 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   for (int i = 0; i < n; ++i) {
     const adapm_block& b = c->blocks[i];
     if (b.mom_mode != ADAPM_MOM_LOWRANK) continue;
-    if (tensor_path_block_ok(*hp, b)) tc_ids.push_back(i);
+    // preconditioned passes exist on the CUDA-core path only
+    if (!hp->inner_precond && tensor_path_block_ok(*hp, b)) tc_ids.push_back(i);
     else if (hp->lowrank_path == ADAPM_PATH_TENSOR) { delete c; return ADAPM_EUNSUPPORTED; }
+    else if (hp->inner_precond && b.rank > 4096) { delete c; return ADAPM_EUNSUPPORTED; }
     else lowrank_ids.push_back(i);
   }
   c->n_tensor_blocks = (int64_t)tc_ids.size();
@@ -336,7 +340,7 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     std::vector<int64_t> gram_off(n, 0);
     for (int64_t i : lowrank_ids) {
       gram_off[i] = work_cursor;
-      work_cursor += round_up(4LL * c->blocks[i].rank * c->blocks[i].rank, kStateAlign);
+      work_cursor += round_up((hp->inner_precond ? 6LL : 4LL) * c->blocks[i].rank * c->blocks[i].rank, kStateAlign);
     }
     const float b1 = hp->beta1, a1 = 1.f - hp->beta1;
     int src_base = BASE_STATE; int64_t src_shift = 0;   // where the current iterate lives
@@ -348,8 +352,10 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
     for (int it = 0; it < K_eff; ++it) {
       const float se = (float)etas[it];
       const int64_t dst_shift = c->ws_lr[dst_buf];
-      std::vector<GemmProb> pAB, pG, pU1, pU2;
-      int64_t tAB = 0, tG = 0, tU1 = 0, tU2 = 0;
+      std::vector<GemmProb> pAB, pG, pU1, pU2, pU3;
+      std::vector<InverseJob> inv;
+      int64_t tAB = 0, tG = 0, tU1 = 0, tU2 = 0, tU3 = 0;
+      const bool precond = hp->inner_precond != 0;
       auto push = [](std::vector<GemmProb>& v, GemmProb p, int64_t& tiles) {
         p.tiles_n = (p.N + 63) / 64;
         p.first_tile = tiles;
@@ -388,6 +394,42 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         p.y_base = (int8_t)src_base; p.y_off = Lc; p.syk = r; p.syj = 1;
         p.c_base = BASE_WORK; p.c_off = G3; p.M = r; p.N = r; p.K = m; p.ldc = r; push(pG, p, tG);
         p.y_base = BASE_STATE; p.y_off = L0; p.c_off = G4; push(pG, p, tG);
+        if (precond) {
+          // Preconditioned pass: A <- L G1 - a1 A, A <- A - b1 L0 G2 (= dl/dL), L' = L - se A S1 with
+          // S1 = (G1 + d I)^-1; B <- G3 R - a1 B, B <- B - b1 G4 R0 (= dl/dR), R' = R - se S3 B, S3 = (G3 + d I)^-1.
+          const int64_t S1 = G4 + (int64_t)r * r, S3 = S1 + (int64_t)r * r;
+          if (!hold) inv.push_back({G1, S1, r, 0});
+          inv.push_back({G3, S3, r, 0});
+          if (!hold) {
+            reset(); p.x_base = (int8_t)src_base; p.x_off = Lc; p.sxi = r; p.sxk = 1;
+            p.y_base = BASE_WORK; p.y_off = G1; p.syk = r; p.syj = 1;
+            p.c_base = BASE_WORK; p.c_off = Aw; p.M = m; p.N = r; p.K = r; p.ldc = r;
+            p.z1_base = BASE_WORK; p.z1_off = Aw; p.c1 = -a1; push(pU1, p, tU1);
+            reset(); p.x_base = BASE_STATE; p.x_off = L0; p.sxi = r; p.sxk = 1;
+            p.y_base = BASE_WORK; p.y_off = G2; p.syk = r; p.syj = 1;
+            p.c_base = BASE_WORK; p.c_off = Aw; p.M = m; p.N = r; p.K = r; p.ldc = r;
+            p.alpha = -b1; p.beta = 1.f; push(pU2, p, tU2);
+          }
+          reset(); p.x_base = BASE_WORK; p.x_off = Aw; p.sxi = r; p.sxk = 1;
+          p.y_base = BASE_WORK; p.y_off = S1; p.syk = r; p.syj = 1;
+          p.c_base = BASE_WORK; p.c_off = Ld; p.M = m; p.N = r; p.K = r; p.ldc = r;
+          p.alpha = -se; p.z1_base = (int8_t)src_base; p.z1_off = Lc; p.c1 = 1.f;
+          if (hold) { p.K = 0; p.alpha = 0.f; }                                            // L' = L
+          push(pU3, p, tU3);
+          reset(); p.x_base = BASE_WORK; p.x_off = G3; p.sxi = r; p.sxk = 1;
+          p.y_base = (int8_t)src_base; p.y_off = Rc; p.syk = nn; p.syj = 1;
+          p.c_base = BASE_WORK; p.c_off = Bw; p.M = r; p.N = nn; p.K = r; p.ldc = nn;
+          p.z1_base = BASE_WORK; p.z1_off = Bw; p.c1 = -a1; push(pU1, p, tU1);
+          reset(); p.x_base = BASE_WORK; p.x_off = G4; p.sxi = r; p.sxk = 1;
+          p.y_base = BASE_STATE; p.y_off = R0; p.syk = nn; p.syj = 1;
+          p.c_base = BASE_WORK; p.c_off = Bw; p.M = r; p.N = nn; p.K = r; p.ldc = nn;
+          p.alpha = -b1; p.beta = 1.f; push(pU2, p, tU2);
+          reset(); p.x_base = BASE_WORK; p.x_off = S3; p.sxi = r; p.sxk = 1;
+          p.y_base = BASE_WORK; p.y_off = Bw; p.syk = nn; p.syj = 1;
+          p.c_base = BASE_WORK; p.c_off = Rd; p.M = r; p.N = nn; p.K = r; p.ldc = nn;
+          p.alpha = -se; p.z1_base = (int8_t)src_base; p.z1_off = Rc; p.c1 = 1.f; push(pU3, p, tU3);
+          continue;
+        }
         // L' = L - se ( L G1 - b1 L0 G2 - a1 A )
         reset(); p.x_base = (int8_t)src_base; p.x_off = Lc; p.sxi = r; p.sxk = 1;
         p.y_base = BASE_WORK; p.y_off = G1; p.syk = r; p.syj = 1;
@@ -411,8 +453,14 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
         p.c_base = BASE_WORK; p.c_off = Rd; p.M = r; p.N = nn; p.K = r; p.ldc = nn;
         p.alpha = se * b1; p.beta = 1.f; push(pU2, p, tU2);
       }
-      for (auto* pv : {&pAB, &pG, &pU1, &pU2}) {
-        const int64_t tiles = pv == &pAB ? tAB : (pv == &pG ? tG : (pv == &pU1 ? tU1 : tU2));
+      for (auto* pv : {&pAB, &pG, &pU1, &pU2, &pU3}) {
+        if (pv == &pU1 && !inv.empty()) {       // the inverses need the Gram matrices and feed the last update
+          Launch IL{LK_SPD_INVERSE, append_table(c->h_tables, inv), (int64_t)inv.size(), (int64_t)inv.size()};
+          IL.phase = phase;
+          prog.push_back(IL);
+        }
+        if (pv->empty()) continue;
+        const int64_t tiles = pv == &pAB ? tAB : (pv == &pG ? tG : (pv == &pU1 ? tU1 : (pv == &pU2 ? tU2 : tU3)));
         Launch GL{LK_GEMM, append_table(c->h_tables, *pv), (int64_t)pv->size(), tiles};
         GL.phase = phase;
         prog.push_back(GL);
@@ -680,6 +728,8 @@ extern "C" int adapm_step(adapm_ctx* c, void* params, const void* grads, void* s
       case LK_STREAM:
         rc = launch_stream((const StreamBlk*)tab, (const int32_t*)(c->d_tables + L.aux0), L.grid, b, sc, hp.grad_dtype, s);
         break;
+      case LK_SPD_INVERSE:
+        rc = launch_spd_inverse((const InverseJob*)tab, L.n_items, work, hp.precond_damping, c->d_status, s); break;
       case LK_GEMM:
         rc = launch_gemm((const GemmProb*)tab, L.n_items, L.grid, b, hp.grad_dtype, s); break;
       case LK_APPLY_SIMT:
@@ -740,6 +790,7 @@ extern "C" const char* adapm_launch_kind_name(int32_t kind) {
     case LK_TC_COPY: return "tc_copy";
     case LK_STREAM: return "stream_update";
     case LK_GEMM: return "gemm_simt";
+    case LK_SPD_INVERSE: return "spd_inverse";
     case LK_APPLY_SIMT: return "apply_simt";
     case LK_COMMIT: return "commit_copy";
     case LK_TC_CONVERT: return "tc_convert";

@@ -201,6 +201,54 @@ __device__ __forceinline__ float block_sum_1024(float x, float* red) {
   return s;
 }
 
+// (G + delta I)^-1 by Gauss-Jordan elimination without pivoting (the matrix is symmetric positive definite), one
+// CTA per matrix, the matrix in global memory, the pivot row and column of a step in shared memory.
+constexpr int kInverseMaxRank = 4096;
+constexpr float kPrecondFloor = 1e-30f;
+
+__global__ void __launch_bounds__(1024) spd_inverse_kernel(const InverseJob* __restrict__ tab, float* __restrict__ work,
+                                                           float damping, const int32_t* __restrict__ status) {
+  extern __shared__ float piv[];         // [0, r): column k before the step; [r, 2r): row k after its scaling
+  __shared__ float red[32];
+  __shared__ int skip;
+  if (threadIdx.x == 0) skip = *status != 0;
+  __syncthreads();
+  if (skip) return;
+  const InverseJob J = tab[blockIdx.x];
+  const int r = J.r;
+  const float* __restrict__ G = work + J.src_off;
+  float* __restrict__ S = work + J.dst_off;
+  float tr = 0.f;
+  for (int i = threadIdx.x; i < r; i += blockDim.x) tr += G[(int64_t)i * r + i];
+  tr = block_sum_1024(tr, red);
+  const float delta = damping * tr / (float)r + kPrecondFloor;
+  const int64_t total = (int64_t)r * r;
+  for (int64_t e = threadIdx.x; e < total; e += blockDim.x) {
+    const int i = (int)(e / r), j = (int)(e % r);
+    S[e] = G[e] + (i == j ? delta : 0.f);
+  }
+  __syncthreads();
+  float* colk = piv;
+  float* rowk = piv + r;
+  for (int k = 0; k < r; ++k) {
+    for (int i = threadIdx.x; i < r; i += blockDim.x) colk[i] = S[(int64_t)i * r + k];
+    __syncthreads();
+    const float inv_p = 1.f / colk[k];
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+      const float x = (j == k ? 1.f : S[(int64_t)k * r + j]) * inv_p;
+      rowk[j] = x;
+      S[(int64_t)k * r + j] = x;
+    }
+    __syncthreads();
+    for (int64_t e = threadIdx.x; e < total; e += blockDim.x) {
+      const int i = (int)(e / r), j = (int)(e % r);
+      if (i == k) continue;
+      S[e] = (j == k ? 0.f : S[e]) - colk[i] * rowk[j];
+    }
+    __syncthreads();
+  }
+}
+
 // Modified Gram-Schmidt over the columns of L, in order, one CTA per block.  draw = 1: the columns are Gaussian
 // draws first (keyed by seed, block, element).  draw = 0: L already holds the matrix to orthonormalise (g Omega of
 // the data-driven start); a column that keeps less than kRangeDrop of its squared length becomes zero.
@@ -273,6 +321,14 @@ int launch_apply_simt(const ApplyBlk* d_tab, int64_t n_blk, int64_t n_tiles, con
     apply_simt_kernel<true><<<(unsigned)n_tiles, 256, 0, s>>>(d_tab, (int)n_blk, b, sc);
   else
     apply_simt_kernel<false><<<(unsigned)n_tiles, 256, 0, s>>>(d_tab, (int)n_blk, b, sc);
+  ADAPM_LAUNCH_CHECK();
+  return ADAPM_OK;
+}
+
+int launch_spd_inverse(const InverseJob* d_tab, int64_t n_jobs, float* work, float damping, const int32_t* status,
+                       cudaStream_t s) {
+  if (n_jobs <= 0) return ADAPM_OK;
+  spd_inverse_kernel<<<(unsigned)n_jobs, 1024, 2 * kInverseMaxRank * sizeof(float), s>>>(d_tab, work, damping, status);
   ADAPM_LAUNCH_CHECK();
   return ADAPM_OK;
 }

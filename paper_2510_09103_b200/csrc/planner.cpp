@@ -117,4 +117,4 @@ extern "C" const char* adapm_strerror(int code) {
   }
 }
 
-extern "C" int adapm_version(void) { return 200; }
+extern "C" int adapm_version(void) { return 201; }

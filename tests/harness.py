@@ -161,7 +161,9 @@ class ParityRun:
                        clip=f32(hpk["clip"]), inner_iters=hpk["inner_iters"], inner_lr_scale=f32(hpk["inner_lr_scale"]),
                        adam_debias=bool(hpk.get("adam_debias", 0)), correction=bool(hpk.get("correction", 1)),
                        max_grad_norm=(f32(hpk["max_grad_norm"]) if hpk.get("max_grad_norm", 0) > 0 else math.inf),
-                       refresh_period=max(1, int(hpk.get("refresh_period", 0))))
+                       refresh_period=max(1, int(hpk.get("refresh_period", 0))),
+                       inner_precond=bool(hpk.get("inner_precond", 0)),
+                       precond_damping=f32(hpk.get("precond_damping", 1e-3)))
         self.ohp = oh
         self.ostate: Dict[int, O.BlockState] = {}
         self.oW: Dict[int, np.ndarray] = {}

@@ -78,6 +78,9 @@ def test_create_rejects_bad_descriptors_on_the_host():
     assert _create_code([ok], max_grad_norm=float("nan")) == -3
     assert _create_code([ok], tune_stage_k=32) == -3
     assert _create_code([ok], tune_panels=4) == -3
+    assert _create_code([ok], inner_precond=2) == -1
+    assert _create_code([ok], inner_precond=1, precond_damping=-1.0) == -3
+    assert _create_code([ok], inner_precond=1, precond_damping=float("nan")) == -3
 
 
 def test_hparams_struct_matches_the_header():

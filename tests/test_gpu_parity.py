@@ -304,6 +304,29 @@ def test_steps_from_a_data_driven_L0_follow_the_oracle():
             run.close()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("damping", [1e-2, 1e-3])
+def test_preconditioned_passes_follow_the_oracle(dtype, damping):
+    """inner_precond = 1 (scaled gradient descent, a variant that is not in the paper): each derivative of Algorithm 2
+    times the damped inverse of the other factor's Gram matrix.  Six steps on the CUDA-core path, every block, every
+    step.  (The fp32 inverse of a Gram matrix with condition number k carries about k * 2^-24; with these damped,
+    well-conditioned matrices L, R and P agree to 1e-6.)"""
+    w = WL.Workload("precond", [], dtype, "normal", steps=6)
+    blocks = _pack([(96, 160, A.MOM_LOWRANK, 8, A.V_BLOCKMEAN, 1), (200, 64, A.MOM_LOWRANK, 3, A.V_ELEMENT, 0),
+                    (256, 192, A.MOM_LOWRANK, 38, A.V_BLOCKMEAN, 0), (70, 130, A.MOM_LOWRANK, 1, A.V_BLOCKMEAN, 1),
+                    (64, 128, A.MOM_FULL, 0, A.V_BLOCKMEAN, 1)])
+    worst = _run(w, True, 6, blocks=blocks, hp=dict(inner_precond=1, precond_damping=damping, inner_lr_scale=0.5))
+    assert max(worst["L"], worst["R"], worst["P"]) <= 1e-4       # seen: 1e-6
+
+
+def test_preconditioned_passes_with_a_refresh_period_and_refusal_on_the_tensor_path():
+    w = WL.Workload("precond", [], "bf16", "normal", steps=5)
+    blocks = _pack([(128, 256, A.MOM_LOWRANK, 12, A.V_BLOCKMEAN, 1), (256, 64, A.MOM_LOWRANK, 5, A.V_BLOCKMEAN, 1)])
+    _run(w, True, 5, blocks=blocks, hp=dict(inner_precond=1, precond_damping=1e-2, inner_lr_scale=0.5, refresh_period=3))
+    with pytest.raises(A.AdapmError):
+        A.adapm_create(blocks, A.hparams(inner_precond=1, lowrank_path=A.PATH_TENSOR))
+
+
 def test_runs_are_bitwise_reproducible_and_resumable():
     import torch
     w = WL.get_workload("tiny")
