@@ -399,6 +399,18 @@ def test_step_requires_workspace_and_aligned_pointers():
     with pytest.raises(A.AdapmError) as e:
         ctx.adapm_step(params[1:], grads, state, 1)
     assert e.value.code == -2
+    # the data-driven start: a missing Omega and misaligned buffers are refused on the host
+    omega = torch.zeros(ctx.adapm_init_omega_floats() + 4, device="cuda")
+    assert ctx.adapm_init_omega_floats() == 64 * 4 and ctx.adapm_init_omega_layout(0) == (0, 64 * 4)
+    with pytest.raises(A.AdapmError) as e:
+        ctx.adapm_state_init_from_grads(state, grads, None)
+    assert e.value.code == -1
+    with pytest.raises(A.AdapmError) as e:
+        ctx.adapm_state_init_from_grads(state, grads, omega[1:])
+    assert e.value.code == -2
+    with pytest.raises(A.AdapmError) as e:
+        ctx.adapm_state_init_from_grads(state[1:], grads, omega)
+    assert e.value.code == -2
     ctx.adapm_destroy()
 
 
