@@ -120,8 +120,9 @@ typedef struct {
                               the paper: scaled gradient descent): dl/dL is multiplied from the right
                               by (R R^T + d_R I)^-1 and dl/dR from the left by (L^T L + d_L I)^-1, with
                               d = precond_damping * trace / r + 1e-30; warm start, schedule and the
-                              simultaneous update are Algorithm 2's.  Runs on the CUDA-core path only
-                              (ADAPM_PATH_TENSOR with it: ADAPM_EUNSUPPORTED)                        */
+                              simultaneous update are Algorithm 2's.  On the tensor path the inverses
+                              and the transformed factors L (L^T L + d I)^-1 and (R R^T + d I)^-1 R come
+                              from CUDA-core kernels before each pass's tensor launches              */
   float   precond_damping; /* >= 0; used when inner_precond = 1                                    */
 } adapm_hparams;
 

@@ -142,7 +142,8 @@ enum LaunchKind : int32_t {
   LK_REDUCE_ROWS,       // reduce_final over the row sums of g^2 that the first refit pass left
   LK_GRADNORM,          // global gradient norm and the clip factor
   LK_TC_COPY,           // previous split copy of L -> final set (steps that hold L)
-  LK_SPD_INVERSE        // damped inverses of the r x r Gram matrices (preconditioned passes)
+  LK_SPD_INVERSE,       // damped inverses of the r x r Gram matrices (preconditioned passes)
+  LK_TC_CONVERT_WORK    // split copy of fp32 arrays that live in the workspace (the transformed factors)
 };
 // when a launch of the program runs
 enum LaunchWhen : int32_t {

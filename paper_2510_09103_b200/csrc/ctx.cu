@@ -108,8 +108,7 @@ extern "C" int adapm_create(const adapm_block* blocks, int64_t n_blocks, const a
   for (int i = 0; i < n; ++i) {
     const adapm_block& b = c->blocks[i];
     if (b.mom_mode != ADAPM_MOM_LOWRANK) continue;
-    // preconditioned passes exist on the CUDA-core path only
-    if (!hp->inner_precond && tensor_path_block_ok(*hp, b)) tc_ids.push_back(i);
+    if (tensor_path_block_ok(*hp, b)) tc_ids.push_back(i);
     else if (hp->lowrank_path == ADAPM_PATH_TENSOR) { delete c; return ADAPM_EUNSUPPORTED; }
     else if (hp->inner_precond && b.rank > 4096) { delete c; return ADAPM_EUNSUPPORTED; }
     else lowrank_ids.push_back(i);
@@ -794,6 +793,7 @@ extern "C" const char* adapm_launch_kind_name(int32_t kind) {
     case LK_APPLY_SIMT: return "apply_simt";
     case LK_COMMIT: return "commit_copy";
     case LK_TC_CONVERT: return "tc_convert";
+    case LK_TC_CONVERT_WORK: return "tc_convert_work";
     case LK_TC_PANEL: return "tc_panel";
     case LK_TC_GRAM: return "tc_gram";
     case LK_TC_APPLY: return "tc_apply";

@@ -48,7 +48,8 @@ enum {
   MAP_W = 24, MAP_G32 = 25, MAP_V = 26,          // W, g, v in quarter-tile boxes (apply)
   MAP_LCAT = 27, MAP_RCAT = 28,                  // X and Y side by side as one matrix (apply)
   MAP_SH = 29,                                   // the bf16 copy of W, boxes like g's (apply; zero without a shadow)
-  kMapsPerBlock = 30
+  MAP_LCN_T = 30, MAP_RTCN_T = 31,               // N side of the transformed factors L S_L and (S_R R)^T (preconditioned passes)
+  kMapsPerBlock = 32
 };
 
 struct ConvertJob {
@@ -130,6 +131,9 @@ struct TcBlock {
   int64_t lc[3], rtc[3], gs[4];    // bf16 element offsets in the workspace; sets 0 = X, 1 = Y, 2 = Z
   int32_t ld[3];                   // row pitch of set s of lc / rtc, in elements
   int64_t rowsum;                  // float offset of the row sums of g^2 in the workspace, or -1
+  // preconditioned passes: split copies of L S_L and (S_R R)^T (pitch 2 half), and in floats the Gram matrices
+  // R R^T, L^T L (gf, gf + r^2), their damped inverses (sf, sf + r^2) and the fp32 products L S_L, S_R R
+  int64_t lct = 0, rtct = 0, gf = 0, sf = 0, ltf = 0, rtf = 0;
 };
 
 struct MapSet {                     // tensor maps for one combination of caller buffers
@@ -374,6 +378,15 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
     t.ld[0] = t.ld[1] = 4 * t.half; t.ld[2] = 2 * t.half;
     for (int w = 0; w < 4; ++w) t.gs[w] = take((int64_t)2 * t.half * 2 * t.half);
     t.rowsum = -1;
+    if (hp.inner_precond) {
+      auto take_f = [&](int64_t floats) { const int64_t off = work_cursor; work_cursor += round_up(floats, kStateAlign); return off; };
+      t.lct = take((int64_t)b.rows * 2 * t.half);
+      t.rtct = take((int64_t)b.cols * 2 * t.half);
+      t.gf = take_f(2LL * b.rank * b.rank);
+      t.sf = take_f(2LL * b.rank * b.rank);
+      t.ltf = take_f((int64_t)b.rows * b.rank);
+      t.rtf = take_f((int64_t)b.rank * b.cols);
+    }
     P->blk.push_back(t);
   }
   P->work_end = work_cursor;
@@ -483,6 +496,60 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
       std::vector<tc::Item> grams, panels;
       std::vector<BlockSpan> spans;
       bool any_sumsq = false;
+      // Preconditioned passes: dl/dL (R R^T + d I)^-1 = (L R - m_t) (S_R R)^T and (L^T L + d I)^-1 dl/dR =
+      // (L S_L)^T (L R - m_t), so the pass is Algorithm 2's with the transformed factors on the N side of every
+      // product.  They are made first, from the fp32 factors in the state (the panels keep those current): the two
+      // Gram matrices and the two products by the batched CUDA-core GEMM, the inverses, then the split copies.
+      const bool precond = hp.inner_precond != 0;
+      if (precond) {
+        std::vector<GemmProb> pG, pT;
+        std::vector<InverseJob> inv;
+        std::vector<ConvertJob> cj;
+        int64_t tG = 0, tT = 0, owners = 0;
+        auto push = [](std::vector<GemmProb>& v, GemmProb p, int64_t& tiles) {
+          p.tiles_n = (p.N + 63) / 64;
+          p.first_tile = tiles;
+          tiles += (int64_t)((p.M + 63) / 64) * p.tiles_n;
+          v.push_back(p);
+        };
+        for (const TcBlock& t : P->blk) {
+          const adapm_block& b = c->blocks[t.id];
+          const int m = b.rows, n = b.cols, r = b.rank;
+          const int64_t L = c->l_off[t.id], R = c->r_off[t.id];
+          const int64_t GR = t.gf, GL = t.gf + (int64_t)r * r, SR = t.sf, SL = t.sf + (int64_t)r * r;
+          GemmProb p;
+          auto reset = [&]() { std::memset(&p, 0, sizeof(p)); p.z1_base = p.z2_base = BASE_NONE; p.alpha = 1.f; };
+          ConvertJob j;
+          std::memset(&j, 0, sizeof(j));
+          j.r = r; j.rp = t.rp; j.half = t.half; j.dst_ld = 2 * t.half;
+          if (!hold) {
+            reset(); p.x_base = BASE_STATE; p.x_off = R; p.sxi = n; p.sxk = 1;             // G_R = R R^T
+            p.y_base = BASE_STATE; p.y_off = R; p.syk = 1; p.syj = n;
+            p.c_base = BASE_WORK; p.c_off = GR; p.M = r; p.N = r; p.K = n; p.ldc = r; push(pG, p, tG);
+            inv.push_back({GR, SR, r, 0});
+            reset(); p.x_base = BASE_WORK; p.x_off = SR; p.sxi = r; p.sxk = 1;              // S_R R
+            p.y_base = BASE_STATE; p.y_off = R; p.syk = n; p.syj = 1;
+            p.c_base = BASE_WORK; p.c_off = t.rtf; p.M = r; p.N = n; p.K = r; p.ldc = n; push(pT, p, tT);
+            j.f32_off = t.rtf; j.own_stride = 1; j.k_stride = n; j.owners = n; j.dst_off = t.rtct;
+            j.first_owner = owners; owners += j.owners; cj.push_back(j);
+          }
+          reset(); p.x_base = BASE_STATE; p.x_off = L; p.sxi = 1; p.sxk = r;                // G_L = L^T L
+          p.y_base = BASE_STATE; p.y_off = L; p.syk = r; p.syj = 1;
+          p.c_base = BASE_WORK; p.c_off = GL; p.M = r; p.N = r; p.K = m; p.ldc = r; push(pG, p, tG);
+          inv.push_back({GL, SL, r, 0});
+          reset(); p.x_base = BASE_STATE; p.x_off = L; p.sxi = r; p.sxk = 1;                // L S_L
+          p.y_base = BASE_WORK; p.y_off = SL; p.syk = r; p.syj = 1;
+          p.c_base = BASE_WORK; p.c_off = t.ltf; p.M = m; p.N = r; p.K = r; p.ldc = r; push(pT, p, tT);
+          j.f32_off = t.ltf; j.own_stride = r; j.k_stride = 1; j.owners = m; j.dst_off = t.lct;
+          j.first_owner = owners; owners += j.owners; cj.push_back(j);
+        }
+        Launch A1{LK_GEMM, append_items(c->h_tables, pG), (int64_t)pG.size(), tG};
+        Launch A2{LK_SPD_INVERSE, append_items(c->h_tables, inv), (int64_t)inv.size(), (int64_t)inv.size()};
+        Launch A3{LK_GEMM, append_items(c->h_tables, pT), (int64_t)pT.size(), tT};
+        Launch A4{LK_TC_CONVERT_WORK, append_items(c->h_tables, cj), (int64_t)cj.size(), (owners + 255) / 256};
+        A4.aux0 = owners;
+        for (Launch* X : {&A1, &A2, &A3, &A4}) { X->when = when; X->phase = phase; prog.push_back(*X); }
+      }
       for (size_t bi = 0; bi < P->blk.size(); ++bi) {
         const TcBlock& t = P->blk[bi];
         const adapm_block& b = c->blocks[t.id];
@@ -516,12 +583,15 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           }
         };
         const int srcL = hold ? prev : src;     // a held L stays in the previous set all step long
+        // the factor on the N side of every product: itself, or its transformed copy in a preconditioned pass
+        const int nR = precond ? mb + MAP_RTCN_T : mb + MAP_RTCN + src;
+        const int nL = precond ? mb + MAP_LCN_T : mb + MAP_LCN + srcL;
         if (!hold) {
-          gram(mb + MAP_RTCT + src, mb + MAP_RTCN + src, n, 0, -1.f / a1);  // Bop1[j][k] = -(R R^T)[j][k] / (1-b1), stored as [k][j]
-          gram(mb + MAP_RTCT + prev, mb + MAP_RTCN + src, n, 1, b1 / a1);   // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
+          gram(mb + MAP_RTCT + src, nR, n, 0, -1.f / a1);  // Bop1[j][k] = -(R R^T)[j][k] / (1-b1), stored as [k][j]
+          gram(mb + MAP_RTCT + prev, nR, n, 1, b1 / a1);   // Bop2[j][k] = b1 (R R0^T)[j][k] / (1-b1)
         }
-        gram(mb + MAP_LCT + srcL, mb + MAP_LCN + srcL, m, 2, -1.f / a1);    // Bop3[j][k] = -(L^T L)[j][k] / (1-b1)
-        gram(mb + MAP_LCT + prev, mb + MAP_LCN + srcL, m, 3, b1 / a1);      // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
+        gram(mb + MAP_LCT + srcL, nL, m, 2, -1.f / a1);    // Bop3[j][k] = -(L^T L)[j][k] / (1-b1)
+        gram(mb + MAP_LCT + prev, nL, m, 3, b1 / a1);      // Bop4[j][k] = b1 (L^T L0)[j][k] / (1-b1)
 
         // one item = up to n_pan adjacent panels of 128 owners that share every B box
         auto panel = [&](bool is_L, int p0, int np) {
@@ -529,8 +599,8 @@ int build_tensor_program(adapm_ctx* c, const std::vector<int64_t>& tc_ids, const
           std::memset(&it, 0, sizeof(it));
           const int mS = (is_L ? mb + MAP_LC : mb + MAP_RTC) + src, m0 = (is_L ? mb + MAP_LC : mb + MAP_RTC) + prev;
           const int g1 = mb + MAP_GS + (is_L ? 0 : 2), g2 = g1 + 1;
-          if (is_L) it.seg[0] = make_seg(geo, mb + MAP_G, 0, p0, 0, np, 0, 128, mb + MAP_RTCN + src, rp, half, n, 0, 2 * rp, 1);  // g R^T
-          else it.seg[0] = make_seg(geo, mb + MAP_GT, p0, 0, 1, np, 128, 0, mb + MAP_LCN + srcL, rp, half, m, 0, 2 * rp, 1);      // g^T L
+          if (is_L) it.seg[0] = make_seg(geo, mb + MAP_G, 0, p0, 0, np, 0, 128, nR, rp, half, n, 0, 2 * rp, 1);  // g R^T
+          else it.seg[0] = make_seg(geo, mb + MAP_GT, p0, 0, 1, np, 128, 0, nL, rp, half, m, 0, 2 * rp, 1);      // g^T L
           // [hi | lo] of the current and of the previous factor against the stacked Gram operands
           it.seg[1] = make_seg(geo, mS, 0, p0, 0, np, 0, 128, g1, rp, half, half + rp, 0, 2 * rp, 0);
           it.seg[2] = make_seg(geo, m0, 0, p0, 0, np, 0, 128, g2, rp, half, half + rp, 0, 2 * rp, 0);
@@ -739,6 +809,12 @@ int tensor_prepare_step(adapm_ctx* c, const Bases& b, int64_t t, cudaStream_t s,
     }
     ok = ok && tc::encode_bf16_matrix(&m[MAP_LCAT], work + t2.lc[0] * 2, rows, 4 * half, 4 * half, 128);
     ok = ok && tc::encode_bf16_matrix(&m[MAP_RCAT], work + t2.rtc[0] * 2, cols, 4 * half, 4 * half, 128);
+    if (c->hp.inner_precond) {
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_LCN_T], work + t2.lct * 2, rows, 2 * half, nb, sk);
+      ok = ok && tc::encode_bf16_chunked(&m[MAP_RTCN_T], work + t2.rtct * 2, cols, 2 * half, nb, sk);
+    } else {
+      std::memset(&m[MAP_LCN_T], 0, 2 * sizeof(CUtensorMap));
+    }
     if (b.shadow)
       ok = ok && tc::encode_panel32(&m[MAP_SH], reinterpret_cast<const char*>(b.shadow) + blk.offset * 2, rows, cols, false);
     else
@@ -771,6 +847,13 @@ int run_tensor_launch(adapm_ctx* c, const Launch& L, const Bases& b, const StepS
       ADAPM_CUDA(cudaMemsetAsync((char*)b.p[BASE_WORK] + P->work_begin * 4, 0, (size_t)(P->work_end - P->work_begin) * 4, s));
       tc_convert_kernel<<<(unsigned)L.grid, 256, 0, s>>>((const ConvertJob*)tab, (int)L.n_items, L.aux0,
                                                         (const float*)b.p[BASE_STATE], (uint16_t*)b.p[BASE_WORK],
+                                                        c->d_status);
+      break;
+    case LK_TC_CONVERT_WORK:
+      // the same split copy from fp32 arrays in the workspace (nothing is zeroed: the padding stays as the last
+      // full rebuild left it)
+      tc_convert_kernel<<<(unsigned)L.grid, 256, 0, s>>>((const ConvertJob*)tab, (int)L.n_items, L.aux0,
+                                                        (const float*)b.p[BASE_WORK], (uint16_t*)b.p[BASE_WORK],
                                                         c->d_status);
       break;
     case LK_TC_COPY:
