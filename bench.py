@@ -565,7 +565,7 @@ def main() -> None:
     ap.add_argument("--no-fold", action="store_true", help="row sums of g^2 from a pass of their own")
     ap.add_argument("--max-grad-norm", type=float, default=0.0, help="global gradient-norm clipping threshold (0 = off)")
     ap.add_argument("--precond", action="store_true",
-                    help="preconditioned refit passes (a variant; CUDA-core path only)")
+                    help="preconditioned refit passes (a variant that is not in the paper)")
     ap.add_argument("--refresh-period", type=int, default=0, help="T: refit both factors every T steps (0/1 = every step)")
     ap.add_argument("--shadow", action="store_true", help="also write the bf16 copy of the parameters")
     args = ap.parse_args()
