@@ -28,19 +28,34 @@ __device__ __forceinline__ void tile_mainloop(float (&acc)[4][4], const void* X,
                                               float (*Ys)[TN + 4]) {
   const int t = threadIdx.x;
   const int ty = t >> 4, tx = t & 15;
+  // where this thread's four elements of each operand tile sit (fixed for the whole K loop)
+  int xi[4], xk[4], yj[4], yk[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (sxk == 1) { xk[q] = t & 15; xi[q] = (t >> 4) + 16 * q; } else { xi[q] = t & 63; xk[q] = (t >> 6) + 4 * q; }
+    if (syj == 1) { yj[q] = t & 63; yk[q] = (t >> 6) + 4 * q; } else { yk[q] = t & 15; yj[q] = (t >> 4) + 16 * q; }
+  }
+  // The next tile's elements are asked for before the present tile is multiplied: their round trip to memory
+  // runs under the 256 FMAs per thread of a tile instead of between two tiles.
+  float xr[4], yr[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = i0 + xi[q], k = k0 + xk[q];
+      xr[q] = (i < M && k < K) ? load_operand<BF16G>(X, x_grad, (int64_t)i * sxi + (int64_t)k * sxk) : 0.f;
+      const int j = j0 + yj[q], k2 = k0 + yk[q];
+      yr[q] = (j < N && k2 < K) ? load_operand<BF16G>(Y, y_grad, (int64_t)k2 * syk + (int64_t)j * syj) : 0.f;
+    }
+  };
+  if (K > 0) fetch(0);
   for (int k0 = 0; k0 < K; k0 += TK) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      int ii, kk;
-      if (sxk == 1) { kk = t & 15; ii = (t >> 4) + 16 * q; } else { ii = t & 63; kk = (t >> 6) + 4 * q; }
-      const int i = i0 + ii, k = k0 + kk;
-      Xs[kk][ii] = (i < M && k < K) ? load_operand<BF16G>(X, x_grad, (int64_t)i * sxi + (int64_t)k * sxk) : 0.f;
-      int jj, kj;
-      if (syj == 1) { jj = t & 63; kj = (t >> 6) + 4 * q; } else { kj = t & 15; jj = (t >> 4) + 16 * q; }
-      const int j = j0 + jj, k2 = k0 + kj;
-      Ys[kj][jj] = (j < N && k2 < K) ? load_operand<BF16G>(Y, y_grad, (int64_t)k2 * syk + (int64_t)j * syj) : 0.f;
+      Xs[xk[q]][xi[q]] = xr[q];
+      Ys[yk[q]][yj[q]] = yr[q];
     }
     __syncthreads();
+    if (k0 + TK < K) fetch(k0 + TK);
 #pragma unroll
     for (int kk = 0; kk < TK; ++kk) {
       const float4 a = *reinterpret_cast<const float4*>(&Xs[kk][ty * 4]);
@@ -67,7 +82,7 @@ __device__ __forceinline__ const T& find_by_first_tile(const T* tab, int n, int6
 }
 
 template <bool BF16G>
-__global__ void __launch_bounds__(256) gemm_kernel(const GemmProb* __restrict__ tab, int n_prob, Bases b) {
+__global__ void __launch_bounds__(256, 3) gemm_kernel(const GemmProb* __restrict__ tab, int n_prob, Bases b) {
   __shared__ __align__(16) float Xs[TK][TM + 4];
   __shared__ __align__(16) float Ys[TK][TN + 4];
   __shared__ GemmProb sP;
